@@ -1,0 +1,190 @@
+/*
+ * structkv.h -- C ABI of the B200 (sm_100a) StructKV prefill-time KV-compression hot path.
+ *
+ * The library scores the observation-window queries of one layer against all prompt keys,
+ * accumulates the per-token in-degree across depth into the Global In-Degree Centrality,
+ * produces the per-layer attention statistics that drive Dynamic Pivot Detection, selects
+ * token budgets (top-k union window) and compacts K/V, hidden states and position ids.
+ *
+ * Conventions
+ *   - Every pointer marked "device" is a CUDA device pointer owned by the caller; "host"
+ *     pointers are ordinary host memory.  The library allocates no device memory: the
+ *     caller passes one workspace at context creation (structkv_workspace_bytes()).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All
+ *     calls enqueue work on it and return without synchronising, except structkv_pivot and
+ *     structkv_poll_device_status, which synchronise that stream.
+ *   - Every call returns a status; invalid arguments are rejected on the host before any
+ *     launch.  There is no CPU fallback: an unsupported shape returns
+ *     STRUCTKV_ERR_UNSUPPORTED.  Device-side waits are bounded; if one expires the kernel
+ *     records STRUCTKV_ERR_TIMEOUT in a device status word read by
+ *     structkv_poll_device_status().
+ *   - A context serialises its calls through its workspace: calls on one context must be
+ *     issued on one stream (or be ordered by the caller).  Distinct contexts are independent.
+ *   - Results are deterministic: the same inputs give the same bits.
+ *
+ * Index conventions: N = n_keys prompt tokens, w = window (the last w positions are the
+ * observation-window queries, row i sits at position t = N-w+i and attends to keys j <= t),
+ * H query heads, H_kv KV heads, G = H / H_kv, head h reads KV head h / G, d = head_dim.
+ */
+#ifndef STRUCTKV_H_
+#define STRUCTKV_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  STRUCTKV_OK = 0,
+  STRUCTKV_ERR_INVALID_ARG = 1, /* null pointer, size out of range, misaligned pointer or stride */
+  STRUCTKV_ERR_UNSUPPORTED = 2, /* shape or dtype outside the supported set */
+  STRUCTKV_ERR_WORKSPACE = 3,   /* workspace missing or too small */
+  STRUCTKV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
+  STRUCTKV_ERR_TIMEOUT = 5      /* a bounded device-side wait expired */
+} structkv_status;
+
+typedef enum { STRUCTKV_BF16 = 0, STRUCTKV_FP32 = 1 } structkv_dtype;
+
+/* Flags of structkv_score_layer. */
+#define STRUCTKV_FLAG_NO_HEAD_STATS 1u /* skip Eq. 5-6: metrics_out[1..2] are written as NaN */
+#define STRUCTKV_FLAG_FORCE_SIMT 2u    /* use the CUDA-core scorer even where the tensor-core one applies */
+
+typedef struct {
+  int n_q_heads;        /* H, a multiple of n_kv_heads */
+  int n_kv_heads;       /* H_kv */
+  int head_dim;         /* d: 64 or 128 */
+  int window;           /* w: 1..256 */
+  int max_seq;          /* largest n_keys any call will pass */
+  structkv_dtype dtype; /* storage type of q_window and k */
+} structkv_config;
+
+typedef struct structkv_ctx structkv_ctx; /* opaque, host-side */
+
+/* Library version (major*10000 + minor*100 + patch). */
+int structkv_version(void);
+
+/* Static, human-readable name of a status code. */
+const char* structkv_status_string(structkv_status s);
+
+/* Bytes of device workspace a context for `cfg` needs (0 if cfg is invalid). */
+size_t structkv_workspace_bytes(const structkv_config* cfg);
+
+/* Creates a context on the current CUDA device.  `workspace_dev` (device, 256-byte aligned,
+ * at least structkv_workspace_bytes(cfg) bytes) stays owned by the caller and must outlive
+ * the context.  The call zeroes the device status word on the default stream and synchronises.
+ * Errors: INVALID_ARG (null pointers, bad config), UNSUPPORTED (head_dim, window),
+ * WORKSPACE (too small / misaligned), CUDA. */
+structkv_status structkv_create(structkv_ctx** ctx_out, const structkv_config* cfg,
+                                void* workspace_dev, size_t workspace_bytes);
+
+/* Frees the host-side context (never touches the workspace). NULL is allowed. */
+void structkv_destroy(structkv_ctx* ctx);
+
+/*
+ * One layer of observation-window scoring.
+ *
+ * Paper: Section 3.2, Eq. 1 (window attention weights a_{t,j} = softmax over keys of
+ * q_t.k_j * scale, causal), Eq. 2 (local saliency S_j = (1/w) sum over window rows and over
+ * all query heads of a_{t,j}), Eq. 3 / Algorithm 1 line 6 (C <- lambda*C + S), and Section
+ * 3.3, Eq. 4 (attention entropy, natural log, mean over heads and window rows), Eq. 5
+ * (sparsity: mean over heads of the mass of the floor(0.1 N) largest entries of the
+ * window-pooled per-head attention) and Eq. 6 (variance: mean over heads of the population
+ * variance over keys of that pooled vector).
+ *
+ *   q_window      device, [H, w, d] contiguous, dtype of the config; positional encoding
+ *                 already applied.  16-byte aligned.
+ *   k             device, element (g, j, c) at k + g*k_stride_head + j*k_stride_token + c
+ *                 (strides in elements; d contiguous).  Base 16-byte aligned, strides
+ *                 multiples of 16 bytes.  Read-only; V is never read.
+ *   n_keys        N, window <= N <= max_seq.
+ *   scale         logit scale (1/sqrt(d), times any temperature the caller folds in).
+ *   lambda        decay of Eq. 3; used only if c_inout != NULL.
+ *   s_out         device, [N] fp32, required: S^(l).
+ *   c_inout       device, [N] fp32 or NULL: updated in place, C <- lambda*C + S.
+ *   head_cols_out device, [H, N] fp32 or NULL: pooled per-head attention
+ *                 abar^(h)_j = (1/w) sum_i a_{i,j} (each row sums to 1).
+ *   metrics_out   device, [3] fp32, required: {entropy, sparsity, variance}.
+ *   flags         STRUCTKV_FLAG_*.
+ *
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, const void* k,
+                                     long long k_stride_head, long long k_stride_token, int n_keys,
+                                     float scale, float lambda, float* s_out, float* c_inout,
+                                     float* head_cols_out, float* metrics_out, unsigned flags,
+                                     void* stream);
+
+/*
+ * Dynamic Pivot Detection.  Paper: Section 3.3, Eq. 7 (first differences of each metric over
+ * layers l = 1..L-1, min-max normalised to [0,1]; a metric with zero range contributes 0),
+ * Eq. 8 (T_l = w1*grad(-entropy) + w2*grad(sparsity) + w3*grad(variance)), Eq. 9 with
+ * Algorithm 1 line 8: the pivot is the layer l in [1, L-1] with the largest T_l (first maximum
+ * wins), capped at l_limit.  NaN sparsity/variance columns (head statistics disabled) count
+ * as constant.  Evaluated in double precision on the host.
+ *
+ *   metrics_dev device, [n_layers, 3] fp32 rows as written by structkv_score_layer.
+ *   weights     host, {w1, w2, w3}.
+ *   l_limit     cap on the pivot, or -1 for none.
+ *   pivot_out   host, receives L* (0 if n_layers < 2).
+ *   t_out       host, [n_layers] or NULL: receives T_l (T_0 = 0).
+ *
+ * Synchronises `stream`.  Errors: INVALID_ARG, CUDA.
+ */
+structkv_status structkv_pivot(structkv_ctx* ctx, const float* metrics_dev, int n_layers,
+                               const float* weights, int l_limit, int* pivot_out, float* t_out,
+                               void* stream);
+
+/*
+ * Global In-Degree Centrality at a known pivot.  Paper: Eq. 3,
+ * c_out[j] = sum_{l=0..pivot} lambda^(pivot-l) * s_hist[l*row_stride + j], evaluated as the
+ * recursion of Algorithm 1 line 6.
+ *
+ *   s_hist device, fp32 rows of length >= n, row_stride in elements;  c_out device, [n] fp32.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_accumulate(structkv_ctx* ctx, const float* s_hist, long long row_stride,
+                                    int pivot, int n, float lambda, float* c_out, void* stream);
+
+/*
+ * Budgeted token selection.  Paper: Eq. 10 (I_struct = top-k(C) union I_win) and Eq. 13
+ * (I_KV = top-k(S^(l)) union I_win), Algorithm 1 lines 10 and 16.  For each of `batch` score
+ * vectors: the (budget - window) highest-scoring tokens of the prefix [0, n - window), ties
+ * to the lower index, written in ascending position order, followed by the window positions
+ * n-window .. n-1.  Scores must not be NaN.
+ *
+ *   scores  device, fp32, vector b starts at scores + b*row_stride (elements).
+ *   idx_out device, [batch, budget] int32.
+ *   window <= budget <= n.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_select(structkv_ctx* ctx, const float* scores, long long row_stride,
+                                int batch, int n, int budget, int window, int* idx_out,
+                                void* stream);
+
+/*
+ * Row gather / compaction.  Paper: Algorithm 1 line 17 (cache K, V at I_KV), line 13 and
+ * Eq. 11-12 (hidden states and position ids at I_struct).  For every slab s and output row r:
+ * dst[s, r, 0:row_bytes] = src[s*slab_stride_bytes + idx[r]*row_stride_bytes + 0:row_bytes],
+ * a byte-exact copy.
+ *
+ *   src   device; dst device, [n_slabs, n_idx, row_bytes] contiguous; they must not overlap.
+ *   idx   device, [n_idx] int32, each in [0, n_rows_src); an out-of-range index copies
+ *         nothing for that row and records STRUCTKV_ERR_INVALID_ARG in the device status word.
+ *   row_bytes > 0.  When src, dst, both strides and row_bytes are multiples of 16 the copy
+ *   uses 16-byte accesses; otherwise 4-byte or single-byte accesses.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long slab_stride_bytes,
+                                 long long row_stride_bytes, int row_bytes, int n_slabs,
+                                 int n_rows_src, const int* idx, int n_idx, void* dst,
+                                 void* stream);
+
+/* Reads and clears the device status word (bounded-wait expiry, bad gather index).
+ * Synchronises `stream`.  Returns STRUCTKV_OK if nothing was recorded. */
+structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STRUCTKV_H_ */

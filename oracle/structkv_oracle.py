@@ -48,7 +48,7 @@ import numpy as np
 
 PAPER_WEIGHTS = (0.2, 0.3, 0.5)      # {w1, w2, w3}, Section 4.1 implementation details
 PAPER_LAMBDA = 0.9                   # decay of the global centrality, same paragraph
-SPARSITY_FRACTION = 0.1              # k = 0.1 N in Eq. 5
+SPARSITY_DENOMINATOR = 10            # k = 0.1 N in Eq. 5, rounded down
 
 
 # --------------------------------------------------------------------------- Eq. 1
@@ -96,7 +96,7 @@ def score_layer(q_win: np.ndarray, k: np.ndarray, scale: float) -> Dict[str, np.
             term = np.where(a > 0.0, a * np.log(a), 0.0)
         row_entropy[h] = -term.sum(axis=1)
     S = head_cols.sum(axis=0)
-    k_rho = max(1, int(np.floor(SPARSITY_FRACTION * N)))
+    k_rho = max(1, N // SPARSITY_DENOMINATOR)
     top_mass = np.sort(head_cols, axis=1)[:, ::-1][:, :k_rho].sum(axis=1)
     return {
         "S": S,

@@ -1,0 +1,174 @@
+"""Thin ctypes binding over the C-ABI library ``libstructkv.so``.
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  PyTorch tensors supply device memory and streams.  Importing this
+module raises if the library has not been built
+(``python -m paper_2604_06746_b200.build``): there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstructkv.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2604_06746_b200.build` "
+        "(the StructKV hot path has no non-CUDA fallback)")
+
+lib = ctypes.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+BF16, FP32 = 0, 1
+FLAG_NO_HEAD_STATS = 1
+FLAG_FORCE_SIMT = 2
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int), ("n_kv_heads", ctypes.c_int),
+                ("head_dim", ctypes.c_int), ("window", ctypes.c_int),
+                ("max_seq", ctypes.c_int), ("dtype", ctypes.c_int)]
+
+
+_vp, _ll, _i, _f, _u = ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_float, ctypes.c_uint
+lib.structkv_version.restype = _i
+lib.structkv_version.argtypes = []
+lib.structkv_status_string.restype = ctypes.c_char_p
+lib.structkv_status_string.argtypes = [_i]
+lib.structkv_workspace_bytes.restype = ctypes.c_size_t
+lib.structkv_workspace_bytes.argtypes = [ctypes.POINTER(Config)]
+lib.structkv_create.restype = _i
+lib.structkv_create.argtypes = [ctypes.POINTER(_vp), ctypes.POINTER(Config), _vp, ctypes.c_size_t]
+lib.structkv_destroy.restype = None
+lib.structkv_destroy.argtypes = [_vp]
+lib.structkv_score_layer.restype = _i
+lib.structkv_score_layer.argtypes = [_vp, _vp, _vp, _ll, _ll, _i, _f, _f, _vp, _vp, _vp, _vp, _u, _vp]
+lib.structkv_pivot.restype = _i
+lib.structkv_pivot.argtypes = [_vp, _vp, _i, ctypes.POINTER(_f), _i, ctypes.POINTER(_i),
+                               ctypes.POINTER(_f), _vp]
+lib.structkv_accumulate.restype = _i
+lib.structkv_accumulate.argtypes = [_vp, _vp, _ll, _i, _i, _f, _vp, _vp]
+lib.structkv_select.restype = _i
+lib.structkv_select.argtypes = [_vp, _vp, _ll, _i, _i, _i, _i, _vp, _vp]
+lib.structkv_compact.restype = _i
+lib.structkv_compact.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _i, _vp, _i, _vp, _vp]
+lib.structkv_poll_device_status.restype = _i
+lib.structkv_poll_device_status.argtypes = [_vp, _vp]
+
+
+class StructKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.structkv_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise StructKVError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def version() -> int:
+    return lib.structkv_version()
+
+
+def workspace_bytes(cfg: Config) -> int:
+    return lib.structkv_workspace_bytes(ctypes.byref(cfg))
+
+
+class Context:
+    """Owns the library context and (through torch) its device workspace."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, max_seq: int,
+                 dtype: torch.dtype, device: str = "cuda:0"):
+        code = {torch.bfloat16: BF16, torch.float32: FP32}[dtype]
+        self.cfg = Config(n_q_heads, n_kv_heads, head_dim, window, max_seq, code)
+        self.device = torch.device(device)
+        self.dtype = dtype
+        self._h = _vp()
+        nbytes = workspace_bytes(self.cfg)
+        if nbytes == 0:
+            raise StructKVError(ERR_UNSUPPORTED, "structkv_workspace_bytes")
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            _check(lib.structkv_create(ctypes.byref(self._h), ctypes.byref(self.cfg),
+                                       self.workspace.data_ptr(), nbytes), "structkv_create")
+
+    def close(self) -> None:
+        if self._h:
+            lib.structkv_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the four calls of the path (plus the closed-form re-accumulation) ---------------
+    def score_layer(self, q_window: torch.Tensor, k: torch.Tensor, scale: float, s_out: torch.Tensor,
+                    metrics_out: torch.Tensor, c_inout: Optional[torch.Tensor] = None,
+                    lam: float = 0.9, head_cols_out: Optional[torch.Tensor] = None, flags: int = 0,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_score_layer: ``k`` is ``[H_kv, N, d]`` with arbitrary head / token strides."""
+        assert q_window.is_contiguous() and k.stride(2) == 1 and k.dtype == self.dtype == q_window.dtype
+        _check(lib.structkv_score_layer(self._h, q_window.data_ptr(), k.data_ptr(), k.stride(0), k.stride(1),
+                                        k.shape[1], scale, lam, s_out.data_ptr(), _ptr(c_inout),
+                                        _ptr(head_cols_out), metrics_out.data_ptr(), flags,
+                                        _stream(stream)), "structkv_score_layer")
+
+    def pivot(self, metrics: torch.Tensor, weights: Sequence[float] = (0.2, 0.3, 0.5), l_limit: int = -1,
+              stream: Optional[torch.cuda.Stream] = None) -> Tuple[int, list]:
+        """structkv_pivot: ``metrics`` is the device ``[L, 3]`` fp32 table; returns ``(L*, T)``."""
+        assert metrics.is_contiguous() and metrics.dtype == torch.float32
+        L = metrics.shape[0]
+        w = (_f * 3)(*weights)
+        piv = _i(0)
+        T = (_f * L)()
+        _check(lib.structkv_pivot(self._h, metrics.data_ptr(), L, w, l_limit, ctypes.byref(piv), T,
+                                  _stream(stream)), "structkv_pivot")
+        return piv.value, list(T)
+
+    def accumulate(self, s_hist: torch.Tensor, pivot: int, lam: float, c_out: torch.Tensor,
+                   stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check(lib.structkv_accumulate(self._h, s_hist.data_ptr(), s_hist.stride(0), pivot, s_hist.shape[1],
+                                       lam, c_out.data_ptr(), _stream(stream)), "structkv_accumulate")
+
+    def select(self, scores: torch.Tensor, budget: int, window: int, idx_out: torch.Tensor,
+               stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_select over ``scores [batch, n]`` (or ``[n]``) into ``idx_out [batch, budget]`` int32."""
+        s2 = scores if scores.dim() == 2 else scores[None]
+        assert s2.stride(1) == 1 and s2.dtype == torch.float32 and idx_out.dtype == torch.int32
+        assert idx_out.is_contiguous() and idx_out.numel() == s2.shape[0] * budget
+        _check(lib.structkv_select(self._h, s2.data_ptr(), s2.stride(0), s2.shape[0], s2.shape[1], budget,
+                                   window, idx_out.data_ptr(), _stream(stream)), "structkv_select")
+
+    def compact(self, src: torch.Tensor, idx: torch.Tensor, dst: torch.Tensor,
+                stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_compact: ``src [n_slabs, n_rows, row...]`` (row contiguous) -> ``dst [n_slabs, n_idx, row...]``."""
+        assert idx.dtype == torch.int32 and idx.is_contiguous() and dst.is_contiguous()
+        row_elems = 1
+        for s in src.shape[2:]:
+            row_elems *= s
+        es = src.element_size()
+        if src.dim() > 2:
+            assert src[0, 0].is_contiguous()
+        _check(lib.structkv_compact(self._h, src.data_ptr(), src.stride(0) * es, src.stride(1) * es,
+                                    row_elems * es, src.shape[0], src.shape[1], idx.data_ptr(),
+                                    idx.numel(), dst.data_ptr(), _stream(stream)), "structkv_compact")
+
+    def poll_device_status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        return lib.structkv_poll_device_status(self._h, _stream(stream))

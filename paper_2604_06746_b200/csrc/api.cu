@@ -1,0 +1,256 @@
+// C ABI of libstructkv: argument validation, context and workspace bookkeeping, dispatch to
+// the kernels, and the host-side pivot rule (Eq. 7-9).
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+struct structkv_ctx {
+  skv::Ctx c;
+};
+
+namespace skv {
+
+static bool config_ok(const structkv_config& cfg) {
+  if (cfg.n_q_heads <= 0 || cfg.n_kv_heads <= 0 || cfg.n_q_heads % cfg.n_kv_heads != 0) return false;
+  if (cfg.n_q_heads > 1024) return false;
+  if (cfg.window < 1 || cfg.max_seq < cfg.window) return false;
+  if (cfg.dtype != STRUCTKV_BF16 && cfg.dtype != STRUCTKV_FP32) return false;
+  if (cfg.head_dim <= 0) return false;
+  return true;
+}
+static bool config_supported(const structkv_config& cfg) {
+  return (cfg.head_dim == 64 || cfg.head_dim == 128) && cfg.window <= 256;
+}
+
+static int rows_pad_of(const structkv_config& cfg) {
+  const int rows_pg = (cfg.n_q_heads / cfg.n_kv_heads) * cfg.window;
+  return cfg.n_kv_heads * (int)align_up((size_t)rows_pg, kRowBlock);
+}
+
+Workspace carve_workspace(const structkv_config& cfg, void* base) {
+  Workspace w{};
+  char* p = (char*)base;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* r = p ? (void*)(p + off) : nullptr;
+    off += align_up(bytes, 256);
+    return r;
+  };
+  const size_t rows_pad = (size_t)rows_pad_of(cfg);
+  const size_t n_pad = align_up((size_t)cfg.max_seq, kKeyTile);
+  w.status = (int*)take(256);
+  w.row_part = (float4*)take((size_t)kMaxParts * rows_pad * sizeof(float4));
+  w.row_lse2 = (float*)take(rows_pad * sizeof(float));
+  w.row_ent = (float*)take(rows_pad * sizeof(float));
+  w.cols = (float*)take((size_t)cfg.n_q_heads * n_pad * sizeof(float));
+  w.head_part = (float*)take((size_t)cfg.n_q_heads * 4 * sizeof(float));
+  w.bytes = off;
+  return w;
+}
+
+}  // namespace skv
+
+using namespace skv;
+
+extern "C" {
+
+int structkv_version(void) { return 100; }
+
+const char* structkv_status_string(structkv_status s) {
+  switch (s) {
+    case STRUCTKV_OK: return "ok";
+    case STRUCTKV_ERR_INVALID_ARG: return "invalid argument";
+    case STRUCTKV_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case STRUCTKV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case STRUCTKV_ERR_CUDA: return "CUDA call failed";
+    case STRUCTKV_ERR_TIMEOUT: return "bounded device wait expired";
+  }
+  return "unknown status";
+}
+
+size_t structkv_workspace_bytes(const structkv_config* cfg) {
+  if (!cfg || !config_ok(*cfg) || !config_supported(*cfg)) return 0;
+  return carve_workspace(*cfg, nullptr).bytes;
+}
+
+structkv_status structkv_create(structkv_ctx** ctx_out, const structkv_config* cfg,
+                                void* workspace_dev, size_t workspace_bytes) {
+  if (!ctx_out || !cfg) return STRUCTKV_ERR_INVALID_ARG;
+  *ctx_out = nullptr;
+  if (!config_ok(*cfg)) return STRUCTKV_ERR_INVALID_ARG;
+  if (!config_supported(*cfg)) return STRUCTKV_ERR_UNSUPPORTED;
+  const size_t need = carve_workspace(*cfg, nullptr).bytes;
+  if (!workspace_dev || workspace_bytes < need || ((uintptr_t)workspace_dev % 256) != 0)
+    return STRUCTKV_ERR_WORKSPACE;
+  structkv_ctx* ctx = new (std::nothrow) structkv_ctx();
+  if (!ctx) return STRUCTKV_ERR_INVALID_ARG;
+  Ctx& c = ctx->c;
+  c.cfg = *cfg;
+  c.ws = carve_workspace(*cfg, workspace_dev);
+  c.rows = cfg->n_q_heads * cfg->window;
+  c.rows_pad = rows_pad_of(*cfg);
+  c.n_pad = (int)align_up((size_t)cfg->max_seq, kKeyTile);
+  c.tc = nullptr;
+  if (cudaGetDevice(&c.device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess ||
+      cudaMemset(c.ws.status, 0, 256) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    delete ctx;
+    return STRUCTKV_ERR_CUDA;
+  }
+  if (cfg->dtype == STRUCTKV_BF16) {
+    const structkv_status s = tc_create(c);
+    if (s != STRUCTKV_OK) { delete ctx; return s; }
+  }
+  *ctx_out = ctx;
+  return STRUCTKV_OK;
+}
+
+void structkv_destroy(structkv_ctx* ctx) {
+  if (!ctx) return;
+  tc_destroy(ctx->c);
+  delete ctx;
+}
+
+structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, const void* k,
+                                     long long k_stride_head, long long k_stride_token, int n_keys,
+                                     float scale, float lambda, float* s_out, float* c_inout,
+                                     float* head_cols_out, float* metrics_out, unsigned flags,
+                                     void* stream) {
+  if (!ctx || !q_window || !k || !s_out || !metrics_out) return STRUCTKV_ERR_INVALID_ARG;
+  Ctx& c = ctx->c;
+  const structkv_config& cfg = c.cfg;
+  const int esz = cfg.dtype == STRUCTKV_BF16 ? 2 : 4;
+  if (n_keys < cfg.window || n_keys > cfg.max_seq) return STRUCTKV_ERR_INVALID_ARG;
+  if (!std::isfinite(scale) || !std::isfinite(lambda)) return STRUCTKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q_window % 16) || ((uintptr_t)k % 16)) return STRUCTKV_ERR_INVALID_ARG;
+  if (k_stride_token < cfg.head_dim || k_stride_head < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if ((k_stride_token * esz) % 16 || (k_stride_head * esz) % 16) return STRUCTKV_ERR_INVALID_ARG;
+  if (((uintptr_t)s_out % 4) || ((uintptr_t)metrics_out % 4) || ((uintptr_t)c_inout % 4) ||
+      ((uintptr_t)head_cols_out % 4))
+    return STRUCTKV_ERR_INVALID_ARG;
+  if (flags & ~(STRUCTKV_FLAG_NO_HEAD_STATS | STRUCTKV_FLAG_FORCE_SIMT)) return STRUCTKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  ScoreArgs a;
+  a.q = q_window; a.k = k;
+  a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
+  a.n_keys = n_keys; a.scale = scale;
+  a.cols = head_cols_out ? head_cols_out : c.ws.cols;
+  a.col_stride = head_cols_out ? (long long)n_keys : (long long)c.n_pad;
+
+  const bool use_tc = cfg.dtype == STRUCTKV_BF16 && !(flags & STRUCTKV_FLAG_FORCE_SIMT) &&
+                      tc_supported(c, a);
+  int parts = 0;
+  cudaError_t e;
+  e = use_tc ? launch_score_tc(c, a, &parts, 1, st) : launch_score_simt(c, a, &parts, 1, st);
+  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  e = launch_finalize_rows(c, parts, metrics_out, st);
+  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  e = use_tc ? launch_score_tc(c, a, &parts, 2, st) : launch_score_simt(c, a, &parts, 2, st);
+  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  e = launch_reduce_columns(c, a.cols, a.col_stride, n_keys, lambda, s_out, c_inout, st);
+  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  e = (flags & STRUCTKV_FLAG_NO_HEAD_STATS) ? launch_fill_nan_stats(metrics_out, st)
+                                            : launch_head_stats(c, a.cols, a.col_stride, n_keys,
+                                                                metrics_out, st);
+  return e == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_pivot(structkv_ctx* ctx, const float* metrics_dev, int n_layers,
+                               const float* weights, int l_limit, int* pivot_out, float* t_out,
+                               void* stream) {
+  if (!ctx || !metrics_dev || !weights || !pivot_out || n_layers < 1 || n_layers > 65536)
+    return STRUCTKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  std::vector<float> m((size_t)n_layers * 3);
+  if (cudaMemcpyAsync(m.data(), metrics_dev, m.size() * sizeof(float), cudaMemcpyDeviceToHost, st) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return STRUCTKV_ERR_CUDA;
+  std::vector<double> T((size_t)n_layers, 0.0);
+  const double sign[3] = {-1.0, 1.0, 1.0};       // Eq. 8 takes the gradient of -entropy
+  for (int col = 0; col < 3 && n_layers >= 2; ++col) {
+    bool nan_col = false;
+    for (int l = 0; l < n_layers; ++l) nan_col |= std::isnan(m[(size_t)l * 3 + col]);
+    if (nan_col) continue;
+    double lo = INFINITY, hi = -INFINITY;
+    for (int l = 1; l < n_layers; ++l) {
+      const double d = sign[col] * ((double)m[(size_t)l * 3 + col] - (double)m[(size_t)(l - 1) * 3 + col]);
+      lo = d < lo ? d : lo;
+      hi = d > hi ? d : hi;
+    }
+    if (!(hi > lo)) continue;
+    for (int l = 1; l < n_layers; ++l) {
+      const double d = sign[col] * ((double)m[(size_t)l * 3 + col] - (double)m[(size_t)(l - 1) * 3 + col]);
+      T[l] += (double)weights[col] * (d - lo) / (hi - lo);
+    }
+  }
+  int best = 0;
+  if (n_layers >= 2) {
+    best = 1;
+    for (int l = 2; l < n_layers; ++l)
+      if (T[l] > T[best]) best = l;
+    if (l_limit >= 0 && best > l_limit) best = l_limit;
+  }
+  *pivot_out = best;
+  if (t_out)
+    for (int l = 0; l < n_layers; ++l) t_out[l] = (float)T[l];
+  return STRUCTKV_OK;
+}
+
+structkv_status structkv_accumulate(structkv_ctx* ctx, const float* s_hist, long long row_stride,
+                                    int pivot, int n, float lambda, float* c_out, void* stream) {
+  if (!ctx || !s_hist || !c_out || pivot < 0 || n < 1 || row_stride < n || !std::isfinite(lambda))
+    return STRUCTKV_ERR_INVALID_ARG;
+  return launch_accumulate(s_hist, row_stride, pivot, n, lambda, c_out, (cudaStream_t)stream) == cudaSuccess
+             ? STRUCTKV_OK
+             : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_select(structkv_ctx* ctx, const float* scores, long long row_stride,
+                                int batch, int n, int budget, int window, int* idx_out,
+                                void* stream) {
+  if (!ctx || !scores || !idx_out) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch < 1 || n < 1 || window < 0 || window > budget || budget > n) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch > 1 && row_stride < n) return STRUCTKV_ERR_INVALID_ARG;
+  return launch_select(scores, row_stride, batch, n, budget, window, idx_out, (cudaStream_t)stream) ==
+                 cudaSuccess
+             ? STRUCTKV_OK
+             : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long slab_stride_bytes,
+                                 long long row_stride_bytes, int row_bytes, int n_slabs,
+                                 int n_rows_src, const int* idx, int n_idx, void* dst,
+                                 void* stream) {
+  if (!ctx || !src || !dst || !idx) return STRUCTKV_ERR_INVALID_ARG;
+  if (row_bytes < 1 || n_slabs < 0 || n_rows_src < 1 || n_idx < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if (row_stride_bytes < row_bytes || slab_stride_bytes < 0) return STRUCTKV_ERR_INVALID_ARG;
+  const Ctx& c = ctx->c;
+  return launch_compact(src, slab_stride_bytes, row_stride_bytes, row_bytes, n_slabs, n_rows_src, idx,
+                        n_idx, dst, c.ws.status, c.sm_count, (cudaStream_t)stream) == cudaSuccess
+             ? STRUCTKV_OK
+             : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream) {
+  if (!ctx) return STRUCTKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int word = 0;
+  if (cudaMemcpyAsync(&word, ctx->c.ws.status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return STRUCTKV_ERR_CUDA;
+  if (word != 0) {
+    if (cudaMemsetAsync(ctx->c.ws.status, 0, sizeof(int), st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+      return STRUCTKV_ERR_CUDA;
+  }
+  if (word < 0 || word > (int)STRUCTKV_ERR_TIMEOUT) return STRUCTKV_ERR_CUDA;
+  return (structkv_status)word;
+}
+
+}  // extern "C"

@@ -1,0 +1,130 @@
+// Internal declarations shared by the translation units of libstructkv (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "structkv.h"
+
+namespace skv {
+
+constexpr int kKeyTile = 128;        // keys per tile in every scorer
+constexpr int kMaxParts = 160;       // upper bound on key segments per score row
+constexpr int kRowBlock = 256;       // score rows (head, window row) per tensor-core row block
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Device status word values are structkv_status codes; 0 = nothing recorded.
+struct Workspace {
+  int* status;          // [64] ints, word 0 is the status
+  float4* row_part;     // [kMaxParts][rows_pad] (m2, Z, U, unused) partial softmax statistics
+  float* row_lse2;      // [rows_pad] log2-domain log-sum-exp of each score row
+  float* row_ent;       // [rows_pad] entropy of each score row (nats)
+  float* cols;          // [H][n_pad] pooled per-head attention when the caller passes none
+  float* head_part;     // [H][4] per-head {sum of squares, top-k mass}
+  size_t bytes;
+};
+
+struct Ctx {
+  structkv_config cfg;
+  Workspace ws;
+  int device;
+  int sm_count;
+  int rows;             // H * w
+  int rows_pad;         // rows per KV group padded to kRowBlock, times H_kv
+  int n_pad;            // max_seq rounded up to kKeyTile
+  void* tc;             // tensor-core scorer state (tensor maps), owned by score_tc.cu
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carves the workspace; with base == nullptr only the size is computed.
+Workspace carve_workspace(const structkv_config& cfg, void* base);
+
+// ---- launchers (each returns cudaGetLastError() of its launches) -------------------------
+struct ScoreArgs {
+  const void* q;            // [H, w, d]
+  const void* k;
+  long long k_stride_head, k_stride_token;   // elements
+  int n_keys;
+  float scale;
+  float* cols;              // [H][col_stride] pooled per-head attention (output of pass 2)
+  long long col_stride;
+};
+
+// CUDA-core two-pass scorer (fp32 or bf16 storage).  parts_out = key segments per row.
+cudaError_t launch_score_simt(const Ctx& ctx, const ScoreArgs& a, int* parts_out, int pass,
+                              cudaStream_t st);
+
+// Tensor-core (tcgen05) two-pass scorer for bf16 storage.
+bool tc_supported(const Ctx& ctx, const ScoreArgs& a);
+structkv_status tc_create(Ctx& ctx);
+void tc_destroy(Ctx& ctx);
+cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pass, cudaStream_t st);
+
+// Merges the per-segment softmax statistics of every row, writes row_lse2 / row_ent and the
+// layer entropy (metrics[0]).
+cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, float* metrics, cudaStream_t st);
+
+// S_j = sum_h cols[h][j]; optional C <- lambda C + S.
+cudaError_t launch_reduce_columns(const Ctx& ctx, const float* cols, long long col_stride, int n,
+                                  float lambda, float* s_out, float* c_inout, cudaStream_t st);
+
+// Eq. 5-6 from the pooled per-head attention; writes metrics[1], metrics[2].
+cudaError_t launch_head_stats(const Ctx& ctx, const float* cols, long long col_stride, int n,
+                              float* metrics, cudaStream_t st);
+cudaError_t launch_fill_nan_stats(float* metrics, cudaStream_t st);
+
+cudaError_t launch_accumulate(const float* s_hist, long long row_stride, int pivot, int n,
+                              float lambda, float* c_out, cudaStream_t st);
+
+cudaError_t launch_select(const float* scores, long long row_stride, int batch, int n, int budget,
+                          int window, int* idx_out, cudaStream_t st);
+
+cudaError_t launch_compact(const void* src, long long slab_stride, long long row_stride,
+                           int row_bytes, int n_slabs, int n_rows_src, const int* idx, int n_idx,
+                           void* dst, int* status, int sm_count, cudaStream_t st);
+
+// 2^x on the special-function unit (relative error about 2^-22; denormal results flush to 0).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Adds one count per candidate lane to hist[bin]; lanes of a warp that hit the same bin are
+// merged into one shared-memory atomic (the values of one vector crowd into few bins).
+__device__ __forceinline__ void hist_add(unsigned* hist, unsigned bin, bool cand) {
+  const unsigned key = cand ? bin : 0xffffffffu;
+  const unsigned peers = __match_any_sync(0xffffffffu, key);
+  if (cand && (threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
+}
+
+// Called by the 32 lanes of warp 0 after a histogram pass.  Walks the `nb` bins (a multiple of
+// 32) from the top and finds the bin holding the `remaining`-th largest candidate; writes that
+// bin and the rank still wanted inside it.
+__device__ __forceinline__ void radix_pick_from_top(const unsigned* hist, int nb, unsigned remaining,
+                                                    unsigned* sel_bin, unsigned* sel_rem) {
+  const int lane = threadIdx.x & 31, per = nb / 32;
+  unsigned mine = 0;
+  for (int b = 0; b < per; ++b) mine += hist[nb - 1 - (lane * per + b)];
+  unsigned incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  const unsigned before = incl - mine;
+  if (before < remaining && remaining <= incl) {
+    unsigned run = before;
+    for (int b = 0; b < per; ++b) {
+      const int bin = nb - 1 - (lane * per + b);
+      const unsigned c = hist[bin];
+      if (run + c >= remaining) { *sel_bin = (unsigned)bin; *sel_rem = remaining - run; break; }
+      run += c;
+    }
+  }
+}
+
+}  // namespace skv

@@ -1,0 +1,88 @@
+"""Sequencing of the C-ABI calls over one prompt (the control flow of Algorithm 1
+replayed over per-layer tensors): score every layer, detect the pivot, rebuild
+the centrality at the pivot, select both budgets, compact K/V, hidden states
+and position ids.  All arithmetic happens inside the library's kernels; this
+file only owns buffers and call order.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+from . import binding
+
+PAPER_LAMBDA = 0.9
+PAPER_WEIGHTS = (0.2, 0.3, 0.5)
+
+
+class Prefill:
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, window: int,
+                 seq: int, kv_budget: int, struct_budget: int, dtype: torch.dtype,
+                 hidden_dim: int = 0, device: str = "cuda:0", lam: float = PAPER_LAMBDA,
+                 weights: Sequence[float] = PAPER_WEIGHTS, l_limit: int = -1, flags: int = 0,
+                 keep_kv: bool = True):
+        self.L, self.H, self.Hkv, self.d, self.w, self.N = n_layers, n_q_heads, n_kv_heads, head_dim, window, seq
+        self.kv_budget, self.struct_budget = kv_budget, struct_budget
+        self.lam, self.weights, self.l_limit, self.flags = lam, tuple(weights), l_limit, flags
+        self.dtype, self.device = dtype, torch.device(device)
+        self.ctx = binding.Context(n_q_heads, n_kv_heads, head_dim, window, seq, dtype, device)
+        dev = self.device
+        f32, i32 = torch.float32, torch.int32
+        self.s_hist = torch.zeros((n_layers, seq), dtype=f32, device=dev)
+        self.metrics = torch.zeros((n_layers, 3), dtype=f32, device=dev)
+        self.c_running = torch.zeros((seq,), dtype=f32, device=dev)
+        self.c_star = torch.zeros((seq,), dtype=f32, device=dev)
+        self.i_kv = torch.zeros((n_layers, kv_budget), dtype=i32, device=dev)
+        self.i_struct = torch.zeros((struct_budget,), dtype=i32, device=dev)
+        n_kv_out = n_layers if keep_kv else 1
+        self.keep_kv = keep_kv
+        self.k_out = torch.empty((n_kv_out, n_kv_heads, kv_budget, head_dim), dtype=dtype, device=dev)
+        self.v_out = torch.empty_like(self.k_out)
+        self.hidden_out = (torch.empty((struct_budget, hidden_dim), dtype=torch.bfloat16, device=dev)
+                           if hidden_dim else None)
+        self.pos_out = torch.empty((struct_budget,), dtype=i32, device=dev)
+        self.pivot = -1
+        self.transition: List[float] = []
+
+    # -- Algorithm 1 lines 3-6 for one layer
+    def score(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, scale: float,
+              head_cols_out: Optional[torch.Tensor] = None) -> None:
+        if layer == 0:
+            self.c_running.zero_()
+        self.ctx.score_layer(q_win, k, scale, self.s_hist[layer], self.metrics[layer],
+                             c_inout=self.c_running, lam=self.lam, head_cols_out=head_cols_out,
+                             flags=self.flags)
+
+    # -- Algorithm 1 lines 7-10 and 16: pivot, centrality at the pivot, both index sets
+    def detect_and_select(self, n_scored: Optional[int] = None) -> int:
+        L = self.L if n_scored is None else n_scored
+        self.pivot, self.transition = self.ctx.pivot(self.metrics[:L], self.weights, self.l_limit)
+        self.ctx.accumulate(self.s_hist, self.pivot, self.lam, self.c_star)
+        self.ctx.select(self.c_star, self.struct_budget, self.w, self.i_struct)
+        self.ctx.select(self.s_hist[:L], self.kv_budget, self.w, self.i_kv[:L])
+        return self.pivot
+
+    # -- Algorithm 1 line 17 for one layer
+    def compact_kv(self, layer: int, k: torch.Tensor, v: torch.Tensor) -> None:
+        slot = layer if self.keep_kv else 0
+        self.ctx.compact(k, self.i_kv[layer], self.k_out[slot])
+        self.ctx.compact(v, self.i_kv[layer], self.v_out[slot])
+
+    # -- Algorithm 1 line 13
+    def compact_hidden(self, hidden: torch.Tensor, positions: torch.Tensor) -> None:
+        self.ctx.compact(hidden[None], self.i_struct, self.hidden_out[None])
+        self.ctx.compact(positions[None, :, None], self.i_struct, self.pos_out[None, :, None])
+
+    def run(self, layers: Sequence[Dict[str, torch.Tensor]], hidden: Optional[torch.Tensor] = None,
+            positions: Optional[torch.Tensor] = None) -> int:
+        """Whole path over resident per-layer tensors (dicts with q_win, k, v, scale)."""
+        for l, t in enumerate(layers):
+            self.score(l, t["q_win"], t["k"], t["scale"])
+        self.detect_and_select(len(layers))
+        for l, t in enumerate(layers):
+            if "v" in t:
+                self.compact_kv(l, t["k"], t["v"])
+        if hidden is not None:
+            self.compact_hidden(hidden, positions)
+        return self.pivot

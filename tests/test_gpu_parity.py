@@ -1,0 +1,133 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the
+same seeded inputs -- element by element for saliency / centrality / metrics, identical pivot,
+selection under the gap rule, bit-exact compaction."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import structkv_oracle as O
+from paper_2604_06746_b200 import synth
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+# The oracle's best and second-best transition scores must be this far apart for the pivot
+# comparison to be meaningful (metric errors of 2e-3 move a transition score by < 1e-2).
+PIVOT_MARGIN = 0.02
+
+
+@pytest.fixture(scope="module")
+def mods(cuda_device):
+    from paper_2604_06746_b200 import binding, pipeline
+    return binding, pipeline
+
+
+def gpu_layers(wl, pl, device):
+    """Small workloads are drawn on the host (one random stream whatever the device) and copied."""
+    out = []
+    for l in range(wl.n_layers):
+        t = synth.make_layer(wl, pl, l, device="cpu")
+        out.append({k: (v.to(device) if torch.is_tensor(v) else v) for k, v in t.items()})
+    return out
+
+
+def oracle_inputs(layers):
+    return [(synth.to_f64(t["q_win"]), synth.to_f64(t["k"]), t["scale"]) for t in layers]
+
+
+def run_and_compare(mods, wl, device, flags=0, check_hidden=True):
+    binding, pipeline = mods
+    pl = synth.plan(wl)
+    layers = gpu_layers(wl, pl, device)
+    hidden = positions = None
+    if check_hidden:
+        hd = 256
+        g = torch.Generator(device=device); g.manual_seed(7)
+        hidden = torch.randn((wl.seq, hd), generator=g, device=device).to(torch.bfloat16)
+        positions = torch.arange(wl.seq, device=device, dtype=torch.int32) * 3 + 1
+    kv_b, st_b = wl.budget, wl.struct_budget()
+    results = {}
+    for weights in (O.PAPER_WEIGHTS, (1.0, 0.0, 0.0)):
+        pf = pipeline.Prefill(wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq,
+                              kv_b, st_b, synth.torch_dtype(wl.dtype), hidden_dim=256 if check_hidden else 0,
+                              device=device, weights=weights, flags=flags)
+        pf.run(layers, hidden, positions)
+        torch.cuda.synchronize()
+        assert pf.ctx.poll_device_status() == binding.OK
+        results[weights] = pf
+    ora = {w: O.prefill(oracle_inputs(layers), wl.window, kv_b, st_b, weights=w) for w in results}
+
+    for weights, pf in results.items():
+        o = ora[weights]
+        tag = f"{wl.name} weights={weights}"
+        s_hist = pf.s_hist.cpu().numpy()
+        metrics = pf.metrics.cpu().numpy()
+        for l in range(wl.n_layers):
+            P.assert_scores_close(s_hist[l], o["s_hist"][l], f"{tag} S layer {l}")
+            for c, name in enumerate(("entropy", "sparsity", "variance")):
+                P.assert_metric_close(metrics[l, c], o["metrics"][l, c], f"{tag} {name} layer {l}")
+        # pivot: the oracle's own margin must be comfortable, then both sides must agree
+        T = np.sort(o["transition"][1:])[::-1]
+        assert len(T) < 2 or T[0] - T[1] >= PIVOT_MARGIN, f"{tag}: oracle transition margin {T[0] - T[1]}"
+        assert pf.pivot == o["pivot"], tag
+        np.testing.assert_allclose(pf.transition[1:], o["transition"][1:], atol=1e-2)
+        P.assert_scores_close(pf.c_star.cpu().numpy(), o["C"], f"{tag} C*")
+        # running recursion of Algorithm 1 line 6 over all layers
+        P.assert_scores_close(pf.c_running.cpu().numpy(),
+                              O.centrality_recursive(o["s_hist"], pf.lam, wl.n_layers - 1), f"{tag} C running")
+        P.assert_selection_matches(pf.i_struct.cpu().numpy(), o["C"], st_b, wl.window, o["i_struct"],
+                                   f"{tag} I_struct")
+        i_kv = pf.i_kv.cpu().numpy()
+        for l in range(wl.n_layers):
+            P.assert_selection_matches(i_kv[l], o["s_hist"][l], kv_b, wl.window, o["i_kv"][l],
+                                       f"{tag} I_KV layer {l}")
+        # compaction is checked bit for bit against the oracle's gather on the GPU's own index sets
+        for l, t in enumerate(layers):
+            for name, out in (("k", pf.k_out), ("v", pf.v_out)):
+                src = t[name].view(torch.int16 if t[name].element_size() == 2 else torch.int32).cpu().numpy()
+                got = out[l].view(torch.int16 if out.element_size() == 2 else torch.int32).cpu().numpy()
+                assert np.array_equal(got, O.compact(src, i_kv[l])), f"{tag} {name} layer {l}"
+        if check_hidden:
+            idx = pf.i_struct.cpu().numpy()
+            assert np.array_equal(pf.hidden_out.view(torch.int16).cpu().numpy(),
+                                  O.compact(hidden.view(torch.int16).cpu().numpy()[None], idx)[0])
+            assert np.array_equal(pf.pos_out.cpu().numpy(), O.compact(positions.cpu().numpy()[None], idx)[0])
+    return results, ora, pl
+
+
+def test_tiny_fp32_full(mods, cuda_device):
+    wl = synth.WORKLOADS["tiny"]
+    results, ora, pl = run_and_compare(mods, wl, cuda_device)
+    pf = results[(1.0, 0.0, 0.0)]
+    assert pf.pivot == 3
+    hubs = set(pl.hub_positions.tolist())
+    assert hubs <= set(pf.i_struct.cpu().numpy().tolist())
+    s_hist = pf.s_hist.cpu().numpy()
+    np.testing.assert_allclose(s_hist.sum(axis=1), wl.n_q_heads, rtol=1e-4)
+
+
+@pytest.mark.parametrize("name,seq,layers,hubs,budget", [
+    ("llama32k", 4096 + 77, 6, 8, 300),       # ragged length: last key tile is partial
+    ("llama128k", 3000, 5, 8, 200),           # sink + delimiters
+    ("qwen64k", 2500, 5, 8, 400),             # GQA 7, window 128, heavy-tailed norms
+])
+def test_scaled_bf16_workloads_simt(mods, cuda_device, name, seq, layers, hubs, budget):
+    binding, _ = mods
+    wl = synth.WORKLOADS[name].scaled(seq, n_layers=layers, n_hubs=hubs, budgets=(budget,))
+    run_and_compare(mods, wl, cuda_device, flags=binding.FLAG_FORCE_SIMT)
+
+
+def test_results_are_deterministic(mods, cuda_device):
+    binding, pipeline = mods
+    wl = synth.WORKLOADS["tiny"]
+    pl = synth.plan(wl)
+    layers = gpu_layers(wl, pl, cuda_device)
+    outs = []
+    for _ in range(2):
+        pf = pipeline.Prefill(wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq,
+                              wl.budget, wl.struct_budget(), torch.float32, device=cuda_device)
+        pf.run(layers)
+        torch.cuda.synchronize()
+        outs.append((pf.s_hist.clone(), pf.metrics.clone(), pf.i_kv.clone(), pf.i_struct.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
