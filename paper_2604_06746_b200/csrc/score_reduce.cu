@@ -26,9 +26,13 @@ __device__ __forceinline__ float block_sum_1024(float v, float* red) {
 }
 
 // One block.  Row r of group g is valid iff its index inside the group is < rows_pg.
-// Merges `parts` partial (m2, Z, U) triples in segment order:
-//   lse2 = m2 + log2 Z,   entropy = ln2 * (log2 Z - U / Z)            (Eq. 4, one row)
-// and writes the mean entropy over the valid rows to metrics[0].
+// Each of the `parts` key segments left (ref, Z, U) for the row: Z = sum 2^(x - ref),
+// U = sum 2^(x - ref) (x - ref), x = logit * log2(e); ref is any reference the segment chose.
+// With l_p = ref_p + log2 Z_p (the segment's log-sum-exp) and M = max_p l_p:
+//   lse2 = M + log2 sum_p 2^(l_p - M)
+//   mean of (x - M) under the row's softmax = sum_p 2^(l_p - M) (ref_p - M + U_p / Z_p) / sum_p 2^(l_p - M)
+//   entropy = ln2 * (lse2 - M - that mean)                                   (Eq. 4, one row)
+// The mean entropy over the valid rows goes to metrics[0].
 __global__ void __launch_bounds__(kFinalThreads)
 finalize_rows(const float4* __restrict__ row_part, int parts, int rows_pad, int rows_pg_pad,
               int rows_pg, int n_valid, float* __restrict__ row_lse2,
@@ -37,32 +41,27 @@ finalize_rows(const float4* __restrict__ row_part, int parts, int rows_pad, int 
   float ent_sum = 0.f;
   for (int r = threadIdx.x; r < rows_pad; r += kFinalThreads) {
     const bool valid = (r % rows_pg_pad) < rows_pg;
-    float m = -INFINITY, Z = 0.f, U = 0.f;
+    float lse2 = INFINITY, ent = 0.f;        // padded rows: 2^(x - inf) = 0 in pass 2
     if (valid) {
+      float M = -INFINITY;
       for (int p = 0; p < parts; ++p) {
         const float4 v = row_part[(size_t)p * rows_pad + r];
-        if (v.x == -INFINITY) continue;
-        if (v.x > m) {                       // rescale the running triple to the new max
-          if (m != -INFINITY) {
-            const float dm = m - v.x, f = fast_exp2(dm);
-            U = f * fmaf(dm, Z, U);
-            Z = f * Z;
-          }
-          m = v.x;
-          Z += v.y;
-          U += v.z;
-        } else {
-          const float dm = v.x - m, f = fast_exp2(dm);
-          Z = fmaf(f, v.y, Z);
-          U = fmaf(f, fmaf(dm, v.y, v.z), U);
-        }
+        if (v.y > 0.f) M = fmaxf(M, v.x + log2f(v.y));
       }
-    }
-    float lse2 = INFINITY, ent = 0.f;        // padded rows: 2^(x - inf) = 0 in pass 2
-    if (valid && Z > 0.f) {
-      const float lz = log2f(Z);
-      lse2 = m + lz;
-      ent = kLn2 * (lz - U / Z);
+      if (M != -INFINITY) {
+        float Zt = 0.f, Xt = 0.f;
+        for (int p = 0; p < parts; ++p) {
+          const float4 v = row_part[(size_t)p * rows_pad + r];
+          if (v.y > 0.f) {
+            const float wgt = fast_exp2(v.x + log2f(v.y) - M);
+            Zt += wgt;
+            Xt = fmaf(wgt, (v.x - M) + v.z / v.y, Xt);
+          }
+        }
+        const float lz = log2f(Zt);
+        lse2 = M + lz;
+        ent = kLn2 * (lz - Xt / Zt);
+      }
     }
     row_lse2[r] = lse2;
     row_ent[r] = ent;

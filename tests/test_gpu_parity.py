@@ -111,10 +111,27 @@ def test_tiny_fp32_full(mods, cuda_device):
     ("llama128k", 3000, 5, 8, 200),           # sink + delimiters
     ("qwen64k", 2500, 5, 8, 400),             # GQA 7, window 128, heavy-tailed norms
 ])
-def test_scaled_bf16_workloads_simt(mods, cuda_device, name, seq, layers, hubs, budget):
+@pytest.mark.parametrize("force_simt", [False, True], ids=["tensor_core", "cuda_core"])
+def test_scaled_bf16_workloads(mods, cuda_device, name, seq, layers, hubs, budget, force_simt):
     binding, _ = mods
     wl = synth.WORKLOADS[name].scaled(seq, n_layers=layers, n_hubs=hubs, budgets=(budget,))
-    run_and_compare(mods, wl, cuda_device, flags=binding.FLAG_FORCE_SIMT)
+    run_and_compare(mods, wl, cuda_device, flags=binding.FLAG_FORCE_SIMT if force_simt else 0)
+
+
+@pytest.mark.parametrize("H,Hkv,d,w,N,budget", [
+    (4, 2, 64, 32, 700, 100),        # head_dim 64, 64 score rows per group (quarter of a row block)
+    (4, 1, 128, 64, 129, 70),        # one KV head; a single full key tile plus one key
+    (14, 2, 128, 128, 1500, 300),    # 896 rows per group: four row blocks, the last one half full
+    (8, 8, 128, 64, 64, 64),         # N == w: every key is a window key, nothing to select
+    (8, 2, 128, 64, 20000, 64),      # budget == window: only the window is kept
+    (8, 2, 64, 128, 333, 333),       # budget == N: everything is kept
+    (6, 2, 128, 8, 900, 50),         # the paper's default window (served by the CUDA-core scorer)
+])
+def test_shape_edges_bf16(mods, cuda_device, H, Hkv, d, w, N, budget):
+    wl = synth.Workload(f"edge-{H}-{Hkv}-{d}-{w}-{N}", 7, 3, H, Hkv, d, N, w, (budget,), "bf16",
+                        min(4, max(0, N - w - 1)), None, hub_layers=(1,), temperatures=(0.7, 1.0, 1.9),
+                        sink=True)
+    run_and_compare(mods, wl, cuda_device)
 
 
 def test_results_are_deterministic(mods, cuda_device):
