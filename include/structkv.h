@@ -116,6 +116,47 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
                                      void* stream);
 
 /*
+ * structkv_score_layer without a context and without a caller workspace.  The paper has no
+ * counterpart: this entry point exists for integration only.
+ *
+ * Some hosts of this library cannot allocate device memory at the point where they score a
+ * layer: a serving engine that hands all free HBM to its paged KV-cache pool at start-up has
+ * nothing left for cudaMalloc to give, and a step that runs inside a latency budget cannot
+ * afford the device-wide synchronisation an allocation or a free implies.  For them the
+ * scratch the scorer needs (per-segment row statistics, row log-sum-exp, pooled per-head
+ * columns, the status word) lives in one array of STRUCTKV_STATIC_SCRATCH_BYTES that is part
+ * of the library image: every GPU that loads the library holds those bytes until the process
+ * exits, whether this function is called or not.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating routine; inputs and outputs are still the caller's.
+ *
+ * Limit: the configuration must satisfy
+ *     0 < structkv_workspace_bytes(cfg) <= STRUCTKV_STATIC_SCRATCH_BYTES
+ * (a Llama-3-8B shape, 32 query heads, window 64, fits up to max_seq = 16384).  A larger
+ * configuration is refused with STRUCTKV_ERR_WORKSPACE before anything is launched.
+ *
+ * Set-up: the first call on each device (with that device current) resolves the device
+ * address of the array and looks up the tensor-map encoder; it synchronises nothing but
+ * should happen before any stream capture begins.  Later calls on that device only enqueue.
+ *
+ * Sharing: all calls on one device use the same array, and it keeps whatever the previous
+ * call left.  The function re-initialises on `stream` what has to start from zero, so calls
+ * issued one after another on one stream are independent; two calls that can overlap on the
+ * GPU (different streams without an ordering between them, or different host threads) race
+ * on the scratch and give undefined results.  A device-side bounded wait that expires during
+ * this call cannot be polled through this entry point; use a context for that.
+ *
+ * Arguments: `cfg` host pointer; everything else exactly as structkv_score_layer, with
+ * cfg->max_seq >= n_keys.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ */
+#define STRUCTKV_STATIC_SCRATCH_BYTES (8u << 20)
+structkv_status structkv_score_layer_static(const structkv_config* cfg, const void* q_window,
+                                            const void* k, long long k_stride_head,
+                                            long long k_stride_token, int n_keys, float scale,
+                                            float lambda, float* s_out, float* c_inout,
+                                            float* head_cols_out, float* metrics_out,
+                                            unsigned flags, void* stream);
+
+/*
  * Dynamic Pivot Detection.  Paper: Section 3.3, Eq. 7 (first differences of each metric over
  * layers l = 1..L-1, min-max normalised to [0,1]; a metric with zero range contributes 0),
  * Eq. 8 (T_l = w1*grad(-entropy) + w2*grad(sparsity) + w3*grad(variance)), Eq. 9 with

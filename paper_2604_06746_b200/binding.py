@@ -48,6 +48,10 @@ lib.structkv_destroy.restype = None
 lib.structkv_destroy.argtypes = [_vp]
 lib.structkv_score_layer.restype = _i
 lib.structkv_score_layer.argtypes = [_vp, _vp, _vp, _ll, _ll, _i, _f, _f, _vp, _vp, _vp, _vp, _u, _vp]
+lib.structkv_score_layer_static.restype = _i
+lib.structkv_score_layer_static.argtypes = [ctypes.POINTER(Config), _vp, _vp, _ll, _ll, _i, _f, _f, _vp, _vp,
+                                            _vp, _vp, _u, _vp]
+STATIC_SCRATCH_BYTES = 8 << 20
 lib.structkv_pivot.restype = _i
 lib.structkv_pivot.argtypes = [_vp, _vp, _i, ctypes.POINTER(_f), _i, ctypes.POINTER(_i),
                                ctypes.POINTER(_f), _vp]
@@ -87,6 +91,31 @@ def version() -> int:
 
 def workspace_bytes(cfg: Config) -> int:
     return lib.structkv_workspace_bytes(ctypes.byref(cfg))
+
+
+def score_layer_static(n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, max_seq: int,
+                       q_window: torch.Tensor, k: torch.Tensor, scale: float, s_out: torch.Tensor,
+                       metrics_out: torch.Tensor, c_inout: Optional[torch.Tensor] = None, lam: float = 0.9,
+                       head_cols_out: Optional[torch.Tensor] = None, flags: int = 0,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """structkv_score_layer_static: one layer of scoring with no context and no workspace.
+
+    For callers that must not allocate device memory where they score (all HBM already given
+    to a cache pool, or a step that cannot take the synchronisation an allocation implies): the
+    scorer's scratch is a fixed array inside the library, so only configurations whose
+    workspace fits ``STATIC_SCRATCH_BYTES`` are accepted, calls on one device share that array
+    and must not overlap on the GPU, and the first call on a device does a one-time set-up that
+    should precede any stream capture.  The current torch device must be the tensors' device.
+    """
+    code = {torch.bfloat16: BF16, torch.float32: FP32}[q_window.dtype]
+    assert q_window.is_contiguous() and k.stride(2) == 1 and k.dtype == q_window.dtype
+    cfg = Config(n_q_heads, n_kv_heads, head_dim, window, max_seq, code)
+    with torch.cuda.device(q_window.device):
+        _check(lib.structkv_score_layer_static(ctypes.byref(cfg), q_window.data_ptr(), k.data_ptr(),
+                                               k.stride(0), k.stride(1), k.shape[1], scale, lam,
+                                               s_out.data_ptr(), _ptr(c_inout), _ptr(head_cols_out),
+                                               metrics_out.data_ptr(), flags, _stream(stream)),
+               "structkv_score_layer_static")
 
 
 class Context:

@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -254,3 +255,76 @@ structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream) {
 }
 
 }  // extern "C"
+
+// ---- context-free scoring on scratch that is part of the library image --------------------
+// In host code `g_static_scratch` is only a handle for the runtime's symbol table, never a
+// device address: the address is resolved once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[STRUCTKV_STATIC_SCRATCH_BYTES];
+
+namespace skv {
+namespace {
+constexpr int kMaxDevices = 64;
+struct StaticSlot {
+  bool ready = false;
+  void* scratch = nullptr;   // device address of g_static_scratch on this device
+  int sm_count = 0;
+  void* tc = nullptr;        // tensor-map encoder state, kept for the life of the process
+};
+StaticSlot g_static_slots[kMaxDevices];
+std::mutex g_static_mutex;
+
+structkv_status static_slot_for_current_device(int* device_out, StaticSlot** slot_out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return STRUCTKV_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticSlot& s = g_static_slots[dev];
+  if (!s.ready) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return STRUCTKV_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return STRUCTKV_ERR_CUDA;
+    Ctx probe{};
+    const structkv_status st = tc_create(probe);      // host-side only: a driver entry point lookup
+    if (st != STRUCTKV_OK) return st;
+    s.tc = probe.tc;
+    s.scratch = ptr;
+    s.ready = true;
+  }
+  *device_out = dev;
+  *slot_out = &s;
+  return STRUCTKV_OK;
+}
+}  // namespace
+}  // namespace skv
+
+extern "C" structkv_status structkv_score_layer_static(
+    const structkv_config* cfg, const void* q_window, const void* k, long long k_stride_head,
+    long long k_stride_token, int n_keys, float scale, float lambda, float* s_out, float* c_inout,
+    float* head_cols_out, float* metrics_out, unsigned flags, void* stream) {
+  if (!cfg) return STRUCTKV_ERR_INVALID_ARG;
+  if (!config_ok(*cfg)) return STRUCTKV_ERR_INVALID_ARG;
+  if (!config_supported(*cfg)) return STRUCTKV_ERR_UNSUPPORTED;
+  const size_t need = carve_workspace(*cfg, nullptr).bytes;
+  if (need == 0 || need > (size_t)STRUCTKV_STATIC_SCRATCH_BYTES) return STRUCTKV_ERR_WORKSPACE;
+  int dev = -1;
+  StaticSlot* slot = nullptr;
+  const structkv_status st = static_slot_for_current_device(&dev, &slot);
+  if (st != STRUCTKV_OK) return st;
+
+  // A context that lives for this call only, laid over the static scratch.
+  structkv_ctx tmp;
+  Ctx& c = tmp.c;
+  c.cfg = *cfg;
+  c.ws = carve_workspace(*cfg, slot->scratch);
+  c.device = dev;
+  c.sm_count = slot->sm_count;
+  c.rows = cfg->n_q_heads * cfg->window;
+  c.rows_pad = rows_pad_of(*cfg);
+  c.n_pad = (int)align_up((size_t)cfg->max_seq, kKeyTile);
+  c.tc = cfg->dtype == STRUCTKV_BF16 ? slot->tc : nullptr;
+  // The scratch keeps the previous call's contents; the status word must start from zero.
+  if (cudaMemsetAsync(c.ws.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  return structkv_score_layer(&tmp, q_window, k, k_stride_head, k_stride_token, n_keys, scale, lambda,
+                              s_out, c_inout, head_cols_out, metrics_out, flags, stream);
+}
