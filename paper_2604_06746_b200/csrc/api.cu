@@ -149,15 +149,15 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   cudaError_t e;
   e = use_tc ? launch_score_tc(c, a, &parts, 1, st) : launch_score_simt(c, a, &parts, 1, st);
   if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
-  e = launch_finalize_rows(c, parts, metrics_out, st);
-  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  if (!use_tc) {
+    e = launch_finalize_rows(c, parts, st);
+    if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  }
   e = use_tc ? launch_score_tc(c, a, &parts, 2, st) : launch_score_simt(c, a, &parts, 2, st);
   if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
   e = launch_reduce_columns(c, a.cols, a.col_stride, n_keys, lambda, s_out, c_inout, st);
   if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
-  e = (flags & STRUCTKV_FLAG_NO_HEAD_STATS) ? launch_fill_nan_stats(metrics_out, st)
-                                            : launch_head_stats(c, a.cols, a.col_stride, n_keys,
-                                                                metrics_out, st);
+  e = launch_metrics(c, a.cols, a.col_stride, n_keys, !(flags & STRUCTKV_FLAG_NO_HEAD_STATS), metrics_out, st);
   return e == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
 }
 

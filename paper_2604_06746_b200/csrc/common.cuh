@@ -63,18 +63,18 @@ structkv_status tc_create(Ctx& ctx);
 void tc_destroy(Ctx& ctx);
 cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pass, cudaStream_t st);
 
-// Merges the per-segment softmax statistics of every row, writes row_lse2 / row_ent and the
-// layer entropy (metrics[0]).
-cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, float* metrics, cudaStream_t st);
+// Merges the per-segment softmax statistics of every row into row_lse2 / row_ent (used by the
+// CUDA-core scorer; the tensor-core scorer does this at the start of its second pass).
+cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st);
 
 // S_j = sum_h cols[h][j]; optional C <- lambda C + S.
 cudaError_t launch_reduce_columns(const Ctx& ctx, const float* cols, long long col_stride, int n,
                                   float lambda, float* s_out, float* c_inout, cudaStream_t st);
 
-// Eq. 5-6 from the pooled per-head attention; writes metrics[1], metrics[2].
-cudaError_t launch_head_stats(const Ctx& ctx, const float* cols, long long col_stride, int n,
-                              float* metrics, cudaStream_t st);
-cudaError_t launch_fill_nan_stats(float* metrics, cudaStream_t st);
+// metrics[0] from row_ent (Eq. 4); metrics[1..2] from the pooled per-head attention (Eq. 5-6),
+// or NaN when head statistics are disabled.
+cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stride, int n,
+                           bool with_head_stats, float* metrics, cudaStream_t st);
 
 cudaError_t launch_accumulate(const float* s_hist, long long row_stride, int pivot, int n,
                               float lambda, float* c_out, cudaStream_t st);

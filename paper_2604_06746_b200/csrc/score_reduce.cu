@@ -1,7 +1,11 @@
 // Small deterministic reductions around the scorers: row finalisation (log-sum-exp, entropy),
 // column reduction over heads with the centrality update, per-head sparsity / variance, and
 // the closed-form centrality re-accumulation.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace skv {
 namespace {
@@ -25,50 +29,43 @@ __device__ __forceinline__ float block_sum_1024(float v, float* red) {
   return red[32];
 }
 
-// One block.  Row r of group g is valid iff its index inside the group is < rows_pg.
-// Each of the `parts` key segments left (ref, Z, U) for the row: Z = sum 2^(x - ref),
+// One thread per score row.  Row r of group g is valid iff its index inside the group is
+// < rows_pg.  Each of the `parts` key segments left (ref, Z, U) for the row: Z = sum 2^(x - ref),
 // U = sum 2^(x - ref) (x - ref), x = logit * log2(e); ref is any reference the segment chose.
 // With l_p = ref_p + log2 Z_p (the segment's log-sum-exp) and M = max_p l_p:
 //   lse2 = M + log2 sum_p 2^(l_p - M)
 //   mean of (x - M) under the row's softmax = sum_p 2^(l_p - M) (ref_p - M + U_p / Z_p) / sum_p 2^(l_p - M)
 //   entropy = ln2 * (lse2 - M - that mean)                                   (Eq. 4, one row)
-// The mean entropy over the valid rows goes to metrics[0].
-__global__ void __launch_bounds__(kFinalThreads)
+__global__ void __launch_bounds__(256)
 finalize_rows(const float4* __restrict__ row_part, int parts, int rows_pad, int rows_pg_pad,
-              int rows_pg, int n_valid, float* __restrict__ row_lse2,
-              float* __restrict__ row_ent, float* __restrict__ metrics) {
-  __shared__ float red[33];
-  float ent_sum = 0.f;
-  for (int r = threadIdx.x; r < rows_pad; r += kFinalThreads) {
-    const bool valid = (r % rows_pg_pad) < rows_pg;
-    float lse2 = INFINITY, ent = 0.f;        // padded rows: 2^(x - inf) = 0 in pass 2
-    if (valid) {
-      float M = -INFINITY;
+              int rows_pg, float* __restrict__ row_lse2, float* __restrict__ row_ent) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows_pad) return;
+  const bool valid = (r % rows_pg_pad) < rows_pg;
+  float lse2 = INFINITY, ent = 0.f;        // padded rows: 2^(x - inf) = 0 in pass 2
+  if (valid) {
+    float M = -INFINITY;
+    for (int p = 0; p < parts; ++p) {
+      const float4 v = row_part[(size_t)p * rows_pad + r];
+      if (v.y > 0.f) M = fmaxf(M, v.x + log2f(v.y));
+    }
+    if (M != -INFINITY) {
+      float Zt = 0.f, Xt = 0.f;
       for (int p = 0; p < parts; ++p) {
         const float4 v = row_part[(size_t)p * rows_pad + r];
-        if (v.y > 0.f) M = fmaxf(M, v.x + log2f(v.y));
-      }
-      if (M != -INFINITY) {
-        float Zt = 0.f, Xt = 0.f;
-        for (int p = 0; p < parts; ++p) {
-          const float4 v = row_part[(size_t)p * rows_pad + r];
-          if (v.y > 0.f) {
-            const float wgt = fast_exp2(v.x + log2f(v.y) - M);
-            Zt += wgt;
-            Xt = fmaf(wgt, (v.x - M) + v.z / v.y, Xt);
-          }
+        if (v.y > 0.f) {
+          const float wgt = fast_exp2(v.x + log2f(v.y) - M);
+          Zt += wgt;
+          Xt = fmaf(wgt, (v.x - M) + v.z / v.y, Xt);
         }
-        const float lz = log2f(Zt);
-        lse2 = M + lz;
-        ent = kLn2 * (lz - Xt / Zt);
       }
+      const float lz = log2f(Zt);
+      lse2 = M + lz;
+      ent = kLn2 * (lz - Xt / Zt);
     }
-    row_lse2[r] = lse2;
-    row_ent[r] = ent;
-    ent_sum += ent;
   }
-  const float tot = block_sum_1024(ent_sum, red);
-  if (threadIdx.x == 0) metrics[0] = tot / (float)n_valid;
+  row_lse2[r] = lse2;
+  row_ent[r] = ent;
 }
 
 // S_j = sum over heads (fixed order) of cols[h][j];  C_j <- lambda C_j + S_j  (Eq. 2, Eq. 3).
@@ -83,63 +80,114 @@ __global__ void reduce_columns(const float* __restrict__ cols, long long col_str
   if (c_inout) c_inout[j] = fmaf(lambda, c_inout[j], s);
 }
 
-// Per head: sum of squares (Eq. 6) and the mass of the k_rho largest entries (Eq. 5), by a
-// three-level radix select on the fp32 bit patterns (all entries are >= 0, so the unsigned
-// order of the bits is the order of the values).  One block per head; deterministic.
+// Per head: sum of squares (Eq. 6) and the mass of the k_rho largest entries (Eq. 5) of the
+// pooled attention vector.  A cluster of kHsCluster CTAs shares one head; each CTA owns a slice
+// of the keys.  All entries are >= 0, so the unsigned order of the fp32 bit patterns is the
+// order of the values.  Two counting sweeps locate the k_rho-th largest value to 22 bits
+// (histograms are merged in CTA 0 of the cluster through distributed shared memory with
+// integer atomics, so the result does not depend on arrival order):
+//   sweep 1: histogram of bits 30..20 (exponent + 3 mantissa bits); sum of squares
+//   sweep 2: exact sum of the entries above the threshold bin (fixed order) and a histogram of
+//            bits 19..9 of the entries inside it
+// The entries inside the threshold bin are then summed as count x bin midpoint: bins of the
+// second level are 2^-14 wide relative to their value, far inside the metric's tolerance.
+constexpr int kHsCluster = 8;
 constexpr int kHsThreads = 1024;
 constexpr int kHsBins = 2048;
 
-__global__ void __launch_bounds__(kHsThreads)
+__global__ void __cluster_dims__(kHsCluster, 1, 1) __launch_bounds__(kHsThreads)
 head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rho,
            float* __restrict__ head_part) {
-  __shared__ unsigned hist[kHsBins];
+  __shared__ unsigned hist[kHsBins];         // this CTA's counts
+  __shared__ unsigned merged[kHsBins];       // cluster-wide counts (CTA 0's copy is the one used)
   __shared__ float red[33];
+  __shared__ float slots[2 * kHsCluster];    // CTA 0: per-CTA {sum of squares, mass above}
   __shared__ unsigned sel_bin, sel_rem;
-  const float* a = cols + (size_t)blockIdx.x * col_stride;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int head = blockIdx.x / kHsCluster;
+  const float* a = cols + (size_t)head * col_stride;
   const int tid = threadIdx.x;
-  unsigned prefix = 0, prefix_mask = 0, remaining = (unsigned)k_rho;
-  const int shifts[3] = {21, 10, 0};
-  const int widths[3] = {11, 11, 10};
+  const int per = (n + kHsCluster - 1) / kHsCluster;
+  const int lo = rank * per, hi = min(n, lo + per);
+  unsigned* merged0 = cluster.map_shared_rank(merged, 0);
+
+  for (int b = tid; b < kHsBins; b += kHsThreads) { hist[b] = 0; merged[b] = 0; }
+  cluster.sync();
   float sq = 0.f;
-  for (int pass = 0; pass < 3; ++pass) {
-    for (int b = tid; b < kHsBins; b += kHsThreads) hist[b] = 0;
-    __syncthreads();
-    const unsigned bmask = (1u << widths[pass]) - 1u;
-    for (int base = 0; base < n; base += kHsThreads) {      // warp-uniform trip count
-      const int j = base + tid;
-      const float v = (j < n) ? a[j] : 0.f;
-      if (pass == 0) sq = fmaf(v, v, sq);
-      const unsigned u = __float_as_uint(v);
-      const bool cand = (j < n) && ((u & prefix_mask) == prefix);
-      hist_add(hist, (u >> shifts[pass]) & bmask, cand);
-    }
-    __syncthreads();
-    if (tid < 32) radix_pick_from_top(hist, 1 << widths[pass], remaining, &sel_bin, &sel_rem);
-    __syncthreads();
-    prefix |= sel_bin << shifts[pass];
-    prefix_mask |= bmask << shifts[pass];
-    remaining = sel_rem;
-    __syncthreads();
-  }
-  // prefix is the bit pattern of the k_rho-th largest value; `remaining` copies of it are taken.
-  const float thr = __uint_as_float(prefix);
-  float mass = 0.f;
-  for (int j = tid; j < n; j += kHsThreads) {
+  for (int j = lo + tid; j < hi; j += kHsThreads) {
     const float v = a[j];
-    if (__float_as_uint(v) > prefix) mass += v;
+    sq = fmaf(v, v, sq);
+    atomicAdd(&hist[(__float_as_uint(v) >> 20) & 0x7ffu], 1u);
   }
-  const float tot_mass = block_sum_1024(mass, red);
+  __syncthreads();
+  for (int b = tid; b < kHsBins; b += kHsThreads)
+    if (hist[b]) atomicAdd(&merged0[b], hist[b]);
+  cluster.sync();
+  if (tid < 32) radix_pick_from_top(merged0, kHsBins, (unsigned)k_rho, &sel_bin, &sel_rem);
+  __syncthreads();
+  const unsigned b1 = sel_bin, rem1 = sel_rem;
+  cluster.sync();                            // every CTA has read the level-1 counts
+  for (int b = tid; b < kHsBins; b += kHsThreads) { hist[b] = 0; merged[b] = 0; }
+  cluster.sync();
+  float mass = 0.f;
+  for (int j = lo + tid; j < hi; j += kHsThreads) {
+    const float v = a[j];
+    const unsigned u = __float_as_uint(v), top = (u >> 20) & 0x7ffu;
+    if (top > b1) mass += v;
+    else if (top == b1) atomicAdd(&hist[(u >> 9) & 0x7ffu], 1u);
+  }
+  __syncthreads();
+  for (int b = tid; b < kHsBins; b += kHsThreads)
+    if (hist[b]) atomicAdd(&merged0[b], hist[b]);
   const float tot_sq = block_sum_1024(sq, red);
+  const float tot_mass = block_sum_1024(mass, red);
   if (tid == 0) {
-    head_part[blockIdx.x * 4 + 0] = tot_sq;
-    head_part[blockIdx.x * 4 + 1] = fmaf((float)remaining, thr, tot_mass);
+    float* slots0 = cluster.map_shared_rank(slots, 0);
+    slots0[2 * rank] = tot_sq;
+    slots0[2 * rank + 1] = tot_mass;
+  }
+  cluster.sync();
+  if (rank == 0) {
+    if (tid < 32) radix_pick_from_top(merged, kHsBins, rem1, &sel_bin, &sel_rem);
+    __syncthreads();
+    const unsigned b2 = sel_bin, rem2 = sel_rem;
+    // entries of the threshold bin above sub-bin b2, and rem2 entries of sub-bin b2 itself
+    float in_bin = 0.f;
+    for (int b = tid; b < kHsBins; b += kHsThreads) {
+      const float mid = __uint_as_float((b1 << 20) | ((unsigned)b << 9) | 0x100u);
+      const unsigned cnt = (unsigned)b > b2 ? merged[b] : ((unsigned)b == b2 ? rem2 : 0u);
+      in_bin = fmaf((float)cnt, mid, in_bin);
+    }
+    const float tot_in_bin = block_sum_1024(in_bin, red);
+    if (tid == 0) {
+      float s2 = 0.f, m = 0.f;
+      for (int r = 0; r < kHsCluster; ++r) { s2 += slots[2 * r]; m += slots[2 * r + 1]; }
+      head_part[head * 4 + 0] = s2;
+      head_part[head * 4 + 1] = m + tot_in_bin;
+    }
   }
 }
 
-// metrics[1] = mean_h top-mass;  metrics[2] = mean_h (sum_sq / n - 1 / n^2)   (rows sum to 1).
-__global__ void head_stats_final(const float* __restrict__ head_part, int H, int n,
-                                 float* __restrict__ metrics) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+// metrics[0] = mean entropy of the valid score rows (Eq. 4);  metrics[1] = mean_h top-mass
+// (Eq. 5);  metrics[2] = mean_h (sum_sq / n - 1 / n^2) (Eq. 6; rows sum to 1).  With head
+// statistics disabled metrics[1..2] are NaN.  One block, fixed summation order.
+__global__ void __launch_bounds__(kFinalThreads)
+finish_metrics(const float* __restrict__ row_ent, int rows_pad, int rows_pg_pad, int rows_pg,
+               int n_valid, const float* __restrict__ head_part, int H, int n, int with_head_stats,
+               float* __restrict__ metrics) {
+  __shared__ float red[33];
+  float ent = 0.f;
+  for (int r = threadIdx.x; r < rows_pad; r += kFinalThreads)
+    if ((r % rows_pg_pad) < rows_pg) ent += row_ent[r];
+  const float tot = block_sum_1024(ent, red);
+  if (threadIdx.x != 0) return;
+  metrics[0] = tot / (float)n_valid;
+  if (!with_head_stats) {
+    metrics[1] = __int_as_float(0x7fc00000);
+    metrics[2] = __int_as_float(0x7fc00000);
+    return;
+  }
   float rho = 0.f, var = 0.f;
   const float inv_n = 1.f / (float)n;
   for (int h = 0; h < H; ++h) {
@@ -148,11 +196,6 @@ __global__ void head_stats_final(const float* __restrict__ head_part, int H, int
   }
   metrics[1] = rho / (float)H;
   metrics[2] = var / (float)H;
-}
-
-__global__ void fill_nan_stats(float* metrics) {
-  metrics[1] = __int_as_float(0x7fc00000);
-  metrics[2] = __int_as_float(0x7fc00000);
 }
 
 // c_out[j] = sum_{l <= pivot} lambda^(pivot - l) s_hist[l][j], as the recursion c = lambda c + s.
@@ -167,12 +210,12 @@ __global__ void accumulate(const float* __restrict__ s_hist, long long row_strid
 
 }  // namespace
 
-cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, float* metrics, cudaStream_t st) {
+cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st) {
   const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
   const int rows_pg = (ctx.cfg.n_q_heads / ctx.cfg.n_kv_heads) * ctx.cfg.window;
-  finalize_rows<<<1, kFinalThreads, 0, st>>>(ctx.ws.row_part, parts, ctx.rows_pad, rows_pg_pad,
-                                            rows_pg, ctx.rows, ctx.ws.row_lse2, ctx.ws.row_ent,
-                                            metrics);
+  finalize_rows<<<(ctx.rows_pad + 255) / 256, 256, 0, st>>>(ctx.ws.row_part, parts, ctx.rows_pad,
+                                                           rows_pg_pad, rows_pg, ctx.ws.row_lse2,
+                                                           ctx.ws.row_ent);
   return cudaGetLastError();
 }
 
@@ -183,18 +226,21 @@ cudaError_t launch_reduce_columns(const Ctx& ctx, const float* cols, long long c
   return cudaGetLastError();
 }
 
-cudaError_t launch_head_stats(const Ctx& ctx, const float* cols, long long col_stride, int n,
-                              float* metrics, cudaStream_t st) {
-  int k_rho = n / 10;
-  if (k_rho < 1) k_rho = 1;
-  head_stats<<<ctx.cfg.n_q_heads, kHsThreads, 0, st>>>(cols, col_stride, n, k_rho,
-                                                       ctx.ws.head_part);
-  head_stats_final<<<1, 32, 0, st>>>(ctx.ws.head_part, ctx.cfg.n_q_heads, n, metrics);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_fill_nan_stats(float* metrics, cudaStream_t st) {
-  fill_nan_stats<<<1, 1, 0, st>>>(metrics);
+cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stride, int n,
+                           bool with_head_stats, float* metrics, cudaStream_t st) {
+  if (with_head_stats) {
+    int k_rho = n / 10;
+    if (k_rho < 1) k_rho = 1;
+    head_stats<<<ctx.cfg.n_q_heads * kHsCluster, kHsThreads, 0, st>>>(cols, col_stride, n, k_rho,
+                                                                      ctx.ws.head_part);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
+  const int rows_pg = (ctx.cfg.n_q_heads / ctx.cfg.n_kv_heads) * ctx.cfg.window;
+  finish_metrics<<<1, kFinalThreads, 0, st>>>(ctx.ws.row_ent, ctx.rows_pad, rows_pg_pad, rows_pg, ctx.rows,
+                                             ctx.ws.head_part, ctx.cfg.n_q_heads, n, with_head_stats ? 1 : 0,
+                                             metrics);
   return cudaGetLastError();
 }
 

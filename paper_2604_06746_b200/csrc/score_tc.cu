@@ -8,8 +8,11 @@
 // so both reductions are loops inside one thread (no shuffles).  A work unit is (KV group g,
 // row block rb of up to 256 score rows); the key range of a unit is split into `segs` equal
 // segments, one CTA each.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the
-// tensor-memory allocation), warps 2..9 = compute.  Every wait is bounded; on expiry the CTA
-// records STRUCTKV_ERR_TIMEOUT, stops, drains its own copies and frees tensor memory.
+// tensor-memory allocation), warps 2..17 = compute (four per scheduler, so that one warp's
+// tensor-memory load latency hides behind the others' arithmetic).  Pass 2 starts by merging
+// the segments' row statistics into each row's log-sum-exp (and, in segment 0, its entropy).
+// Every wait is bounded; on expiry the CTA records STRUCTKV_ERR_TIMEOUT, stops, drains its
+// own copies and frees tensor memory.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -20,16 +23,17 @@ namespace {
 
 constexpr int kStages = 4;             // K tile ring
 constexpr int kAccStages = 2;          // accumulator ring in tensor memory (256 columns each)
-constexpr int kTcThreads = 320;        // 10 warps
-constexpr int kComputeThreads = 256;
+constexpr int kComputeWarps = 16;
+constexpr int kComputeThreads = kComputeWarps * 32;
+constexpr int kTcThreads = 64 + kComputeThreads;   // TMA warp, MMA warp, compute warps
 constexpr unsigned long long kWaitCycles = 1000000000ull;   // about 0.5 s at the maximum SM clock
 constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 0 * x stays finite
 
 struct TcParams {
   int n_keys, window, group, rows_pg, rows_pg_pad, rows_pad, n_rb, segs, n_tiles;
   float c2;                            // scale * log2(e)
-  float4* row_part;                    // pass 1 out
-  const float* row_lse2;               // pass 2 in
+  float4* row_part;                    // pass 1 out, pass 2 in: [2 * segs][rows_pad] (ref, Z, U, -)
+  float* row_ent;                      // pass 2 out (segment 0 only): entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride]
   long long col_stride;
   int* status;
@@ -111,6 +115,39 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Waits for the thread's outstanding tensor-memory loads.  The loaded registers are operands,
+// so no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(float (&v)[32]) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
+}
+
+// 2^x on the FMA pipe for x in [-125, 126]: round-to-nearest split x = n + f with the
+// 1.5 * 2^23 trick (n lands in the low mantissa bits of t), a degree-3 minimax polynomial
+// for 2^f on [-0.5, 0.5] (relative error 7.5e-5), and n added into the exponent field.
+__device__ __forceinline__ float exp2_poly(float x) {
+  const float t = x + 12582912.0f;
+  const float f = x - (t - 12582912.0f);
+  float p = fmaf(0.0551716685f, f, 0.2426111251f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999280572f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// Of every 8 consecutive elements the first kPoly1 (pass 1) / kPoly2 (pass 2) take the
+// polynomial, the rest the special-function unit.
+#ifndef SKV_POLY1
+#define SKV_POLY1 0
+#endif
+#ifndef SKV_POLY2
+#define SKV_POLY2 0
+#endif
+constexpr int kPoly1 = SKV_POLY1, kPoly2 = SKV_POLY2;
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, 8-row
 // groups 1024 bytes apart (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).
@@ -167,6 +204,9 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   const int t_lo = (int)((long long)seg * p.n_tiles / p.segs);
   const int t_hi = (int)((long long)(seg + 1) * p.n_tiles / p.segs);
   const int n_my = t_hi - t_lo;
+  // Pass 1 sweeps its key tiles forward, pass 2 backward: the tiles pass 1 touched last are
+  // the ones still in L2 when pass 2 starts.
+  auto tile_of = [&](int t) { return PASS == 1 ? t_lo + t : t_hi - 1 - t; };
   const int rows_here = min(kRowBlock, p.rows_pg - rb * kRowBlock);     // valid score rows in this block
   const int n_half = (rows_here + 127) / 128;
 
@@ -175,16 +215,11 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     mbar_init(bars + 8 * kBarQ, 1);
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(bars + 8 * (kBarAccFull + a), 1);
-      mbar_init(bars + 8 * (kBarAccEmpty + a), kComputeThreads);
+      mbar_init(bars + 8 * (kBarAccEmpty + a), kComputeWarps);   // one arrival per compute warp
     }
     mbar_init(bars + 8 * kBarDrain, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (PASS == 2) {
-    // log-sum-exp of the block's rows; padded rows hold +inf so they contribute 2^(-inf) = 0
-    for (int r = threadIdx.x; r < kRowBlock; r += kTcThreads)
-      lse_s[r] = (r < rows_here) ? p.row_lse2[g * p.rows_pg_pad + rb * kRowBlock + r] : INFINITY;
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
@@ -210,7 +245,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         mbar_expect_tx(bars + 8 * (kBarFull + s), L::kKBytes);
         for (int c = 0; c < L::kSub; ++c)
           tma_load_3d(base + L::kKOff + s * L::kKBytes + c * (L::kKBytes / L::kSub), &map_k,
-                      bars + 8 * (kBarFull + s), c * 64, (t_lo + t) * kKeyTile, g);
+                      bars + 8 * (kBarFull + s), c * 64, tile_of(t) * kKeyTile, g);
         ++issued;
       }
       // drain: every copy this thread issued must have landed before the CTA may exit
@@ -222,6 +257,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     // ---------------- MMA issuer ----------------
     if (lane == 0 && n_my > 0) {
       constexpr uint32_t idesc = (PASS == 1) ? instr_desc(128, 128) : instr_desc(128, 256);
+      const uint64_t q_desc0 = smem_desc(base + L::kQOff), k_desc0 = smem_desc(base + L::kKOff);
       bool ok = mbar_wait(bars + 8 * kBarQ, 0, abort_flag);
       int t = 0;
       for (; ok && t < n_my; ++t) {
@@ -229,23 +265,23 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         if (!mbar_wait(bars + 8 * (kBarFull + s), (uint32_t)(t / kStages) & 1u, abort_flag)) break;
         if (!mbar_wait(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(t / kAccStages) & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
-        const uint32_t k_tile = base + L::kKOff + s * L::kKBytes;
-        const uint32_t q_tile = base + L::kQOff;
+        // descriptors differ only in the start-address field (16-byte units, no carry out of it)
+        const uint64_t kd = k_desc0 + (uint64_t)((s * L::kKBytes) >> 4);
         if (PASS == 1) {
           for (int hf = 0; hf < n_half; ++hf) {
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t qa = q_tile + (kk / 4) * (L::kQBytes / L::kSub) + hf * (128 * 128) + (kk % 4) * 32;
-              const uint32_t kb = k_tile + (kk / 4) * (L::kKBytes / L::kSub) + (kk % 4) * 32;
-              tc_mma_bf16(tmem + a * 256 + hf * 128, smem_desc(qa), smem_desc(kb), idesc, kk > 0);
+              const uint32_t qo = (kk / 4) * (L::kQBytes / L::kSub) + hf * (128 * 128) + (kk % 4) * 32;
+              const uint32_t ko = (kk / 4) * (L::kKBytes / L::kSub) + (kk % 4) * 32;
+              tc_mma_bf16(tmem + a * 256 + hf * 128, q_desc0 + (qo >> 4), kd + (ko >> 4), idesc, kk > 0);
             }
           }
         } else {
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t ka = k_tile + (kk / 4) * (L::kKBytes / L::kSub) + (kk % 4) * 32;
-            const uint32_t qb = q_tile + (kk / 4) * (L::kQBytes / L::kSub) + (kk % 4) * 32;
-            tc_mma_bf16(tmem + a * 256, smem_desc(ka), smem_desc(qb), idesc, kk > 0);
+            const uint32_t ko = (kk / 4) * (L::kKBytes / L::kSub) + (kk % 4) * 32;
+            const uint32_t qo = (kk / 4) * (L::kQBytes / L::kSub) + (kk % 4) * 32;
+            tc_mma_bf16(tmem + a * 256, kd + (ko >> 4), q_desc0 + (qo >> 4), idesc, kk > 0);
           }
         }
         tc_commit(bars + 8 * (kBarEmpty + s));       // K stage reusable once these MMAs have read it
@@ -257,158 +293,214 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     }
   } else {
     // ---------------- compute warps ----------------
-    const int cw = warp - 2;                 // 0..7
+    const int cw = warp - 2;                 // 0..15
     const int quarter = warp & 3;            // tensor-memory lane quarter this warp may read
-    const int half = cw >> 2;                // pass 1: row half; pass 2: column half
+    const int sub = cw >> 2;                 // which 64 accumulator columns of a tile this warp reads
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     // a tile is "plain" when all of its keys are visible to every window row (j0 + 127 <= N - w);
     // the first (N - w + 1) / 128 tiles are
     const int first_tail_tile = (p.n_keys - p.window + 1) / kKeyTile;
+    float v[32];
+    // lane 0 polls the barrier for its warp (bounded); the outcome is broadcast
+    auto acc_full = [&](int t) {
+      int ok = 1;
+      if (lane == 0)
+        ok = mbar_wait(bars + 8 * (kBarAccFull + t % kAccStages), (uint32_t)(t / kAccStages) & 1u, abort_flag);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      tc_fence_after();
+      return ok != 0;
+    };
+    // all of this warp's loads of the tile have landed: one arrival per warp frees the accumulator
+    auto acc_release = [&](int t) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * (kBarAccEmpty + t % kAccStages));
+    };
 
     if (PASS == 1) {
+      // accumulator columns [0,128) hold rows 0..127 x the tile's 128 keys, [128,256) rows 128..255;
+      // this thread owns one row and 64 of the tile's keys
+      const int half = sub & 1, ch = sub >> 1;
       const int row_in_block = half * 128 + quarter * 32 + lane;
       const bool row_valid = row_in_block < rows_here;
       const bool warp_active = (half * 128 + quarter * 32) < rows_here;
       const int i_win = (rb * kRowBlock + row_in_block) % p.window;      // window row index of this score row
       const int t_pos = p.n_keys - p.window + i_win;                     // its position: sees keys <= t_pos
       float ref = -INFINITY, Z = 0.f, U = 0.f;
-      for (int t = 0; t < n_my; ++t) {
-        const int a = t % kAccStages;
-        if (!mbar_wait(bars + 8 * (kBarAccFull + a), (uint32_t)(t / kAccStages) & 1u, abort_flag)) break;
-        tc_fence_after();
-        if (warp_active) {
-          const uint32_t taddr = tmem + lane_base + a * 256 + half * 128;
-          const int j0 = (t_lo + t) * kKeyTile;
-          const bool plain = (t_lo + t) < first_tail_tile && t > 0;
-          // Every tensor-memory load below is executed by the whole warp (the instruction is
-          // warp-collective); only the arithmetic on the loaded values is per-thread.
-          bool redo = !plain;
+      // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible
+      auto accumulate = [&]() {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float x = fmaf(v[e], p.c2, -ref);
+          const float pr = ((e & 7) < kPoly1) ? exp2_poly(fminf(fmaxf(x, -125.f), 126.f)) : fast_exp2(x);
+          Z += pr;
+          U = fmaf(pr, x, U);
+        }
+      };
+      // same with the causal mask, moving the reference up to the chunk maximum first
+      // (v[0] is key jb); works from registers, so the accumulator is not needed again
+      auto accumulate_careful = [&](int jb) {
+        float mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (jb + e <= t_pos) mx = fmaxf(mx, v[e] * p.c2);
+        if (mx > ref) {
+          if (ref != -INFINITY) {
+            const float dm = ref - mx, f = fast_exp2(dm);
+            U = f * fmaf(dm, Z, U);
+            Z = f * Z;
+          }
+          ref = mx;
+        }
+        const float ref_use = (ref == -INFINITY) ? 0.f : ref;      // row has seen no key yet: all masked
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float x = (jb + e <= t_pos) ? fmaf(v[e], p.c2, -ref_use) : kMasked;
+          const float pr = fast_exp2(x);
+          Z += pr;
+          U = fmaf(pr, x, U);
+        }
+      };
+      // `fast` is warp-uniform: the tile is unmasked and the reference already exists
+      auto chunk = [&](int jb, bool fast) {
+        if (fast) {
           const float Z0 = Z, U0 = U;
-          if (plain) {
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              float v[32];
-              tmem_ld32(taddr + c * 32, v);
-              tmem_ld_wait();
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const float x = fmaf(v[e], p.c2, -ref);
-                const float pr = fast_exp2(x);
-                Z += pr;
-                U = fmaf(pr, x, U);
-              }
-            }
-            // a logit far above the reference overflowed 2^x: the whole warp re-references the tile
-            const bool ovf = !(Z < 3.0e38f) || !(fabsf(U) < 3.0e38f);
-            redo = __any_sync(0xffffffffu, ovf);
-            if (redo) { Z = Z0; U = U0; }
-          }
-          if (redo) {
-            // masked / first / overflowed tile: find the tile maximum, move the reference, accumulate
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              float v[32];
-              tmem_ld32(taddr + c * 32, v);
-              tmem_ld_wait();
-#pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (j0 + c * 32 + e <= t_pos) mx = fmaxf(mx, v[e] * p.c2);
-            }
-            if (mx > ref) {
-              if (ref != -INFINITY) {
-                const float dm = ref - mx, f = fast_exp2(dm);
-                U = f * fmaf(dm, Z, U);
-                Z = f * Z;
-              }
-              ref = mx;
-            }
-            const float ref_use = (ref == -INFINITY) ? 0.f : ref;    // row has seen no key yet: all masked
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              float v[32];
-              tmem_ld32(taddr + c * 32, v);
-              tmem_ld_wait();
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const float x = (j0 + c * 32 + e <= t_pos) ? fmaf(v[e], p.c2, -ref_use) : kMasked;
-                const float pr = fast_exp2(x);
-                Z += pr;
-                U = fmaf(pr, x, U);
-              }
-            }
-          }
+          accumulate();
+          // a logit far above the reference overflowed (or was clamped at 2^126): redo the chunk
+          const bool ovf = !(Z < 4.0e37f) || !(fabsf(U) < 3.0e38f);
+          if (__any_sync(0xffffffffu, ovf)) { Z = Z0; U = U0; accumulate_careful(jb); }
+        } else {
+          accumulate_careful(jb);
         }
-        tc_fence_before();
-        mbar_arrive(bars + 8 * (kBarAccEmpty + a));
-      }
-      if (row_valid && n_my > 0)
-        p.row_part[(size_t)seg * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
-            make_float4(ref, Z, U, 0.f);
-      else if (row_valid)
-        p.row_part[(size_t)seg * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
-            make_float4(-INFINITY, 0.f, 0.f, 0.f);
-    } else {
-      // pass 2: this thread owns key (tile * 128 + quarter * 32 + lane) and the block's score rows
-      // [half * 128, half * 128 + 128); those rows belong to 128 / W heads (or half of one head).
-      constexpr int kHeads = (W <= 128) ? 128 / W : 1;     // heads per column half
-      constexpr int kChunksPerHead = 4 / kHeads;           // 32-column chunks per head
-      const float inv_w = 1.0f / (float)p.window;
-      const int row0 = rb * kRowBlock + half * 128;        // first local score row of this half
-      const bool half_active = half * 128 < rows_here;
+      };
       for (int t = 0; t < n_my; ++t) {
-        const int a = t % kAccStages;
-        if (!mbar_wait(bars + 8 * (kBarAccFull + a), (uint32_t)(t / kAccStages) & 1u, abort_flag)) break;
-        tc_fence_after();
-        const int j = (t_lo + t) * kKeyTile + quarter * 32 + lane;
-        float acc[kHeads];
-#pragma unroll
-        for (int hh = 0; hh < kHeads; ++hh) acc[hh] = 0.f;
-        if (half_active) {
-          const uint32_t taddr = tmem + lane_base + a * 256 + half * 128;
-          const bool plain = (t_lo + t) < first_tail_tile;
-          const int i_min = j - (p.n_keys - p.window);      // window rows i < i_min do not see key j
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            float v[32];
-            tmem_ld32(taddr + c * 32, v);
-            tmem_ld_wait();
-            const float4* l4 = reinterpret_cast<const float4*>(lse_s + half * 128 + c * 32);
-            float s = 0.f;
-            if (plain) {
-#pragma unroll
-              for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 l = l4[e4];
-                s += fast_exp2(fmaf(v[4 * e4 + 0], p.c2, -l.x));
-                s += fast_exp2(fmaf(v[4 * e4 + 1], p.c2, -l.y));
-                s += fast_exp2(fmaf(v[4 * e4 + 2], p.c2, -l.z));
-                s += fast_exp2(fmaf(v[4 * e4 + 3], p.c2, -l.w));
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const int i = (row0 + c * 32 + e) % p.window;
-                const float x = fmaf(v[e], p.c2, -lse_s[half * 128 + c * 32 + e]);
-                s += (i >= i_min) ? fast_exp2(x) : 0.f;
-              }
+        if (!acc_full(t)) break;
+        const uint32_t taddr = tmem + lane_base + (uint32_t)((t % kAccStages) * 256 + half * 128 + ch * 64);
+        const int jb = (t_lo + t) * kKeyTile + ch * 64;
+        const bool plain = (t_lo + t) < first_tail_tile;
+        if (warp_active) {
+          tmem_ld32(taddr, v);
+          tmem_ld_wait(v);
+          chunk(jb, plain && t > 0);
+          tmem_ld32(taddr + 32, v);
+          tmem_ld_wait(v);
+        }
+        acc_release(t);
+        if (warp_active) chunk(jb + 32, plain);
+      }
+      // two partial statistics per (row, segment): one per 64-key half of the tiles
+      if (row_valid)
+        p.row_part[(size_t)(seg * 2 + ch) * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
+            n_my > 0 ? make_float4(ref, Z, U, 0.f) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
+    } else {
+      // pass 2.  First the compute threads merge the partial statistics of this block's rows:
+      // with l_s = ref_s + log2 Z_s (a partial's log-sum-exp) and M = max_s l_s,
+      //   lse2 = M + log2 sum_s 2^(l_s - M),
+      //   entropy = ln2 (lse2 - M - sum_s 2^(l_s - M) (ref_s - M + U_s / Z_s) / sum_s 2^(l_s - M)).
+      // Padded rows get +inf so that they contribute 2^(-inf) = 0.
+      {
+        const int r = (int)threadIdx.x - 64;
+        if (r < kRowBlock) {
+          float lse2 = INFINITY, ent = 0.f;
+          const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
+          const int parts = 2 * p.segs;
+          if (r < rows_here) {
+            float M = -INFINITY;
+            for (int s = 0; s < parts; ++s) {
+              const float4 pv = p.row_part[(size_t)s * p.rows_pad + row];
+              if (pv.y > 0.f) M = fmaxf(M, pv.x + log2f(pv.y));
             }
-            acc[c / kChunksPerHead] += s;
+            if (M != -INFINITY) {
+              float Zt = 0.f, Xt = 0.f;
+              for (int s = 0; s < parts; ++s) {
+                const float4 pv = p.row_part[(size_t)s * p.rows_pad + row];
+                if (pv.y > 0.f) {
+                  const float wgt = fast_exp2(pv.x + log2f(pv.y) - M);
+                  Zt += wgt;
+                  Xt = fmaf(wgt, (pv.x - M) + pv.z / pv.y, Xt);
+                }
+              }
+              const float lz = log2f(Zt);
+              lse2 = M + lz;
+              ent = kLn2 * (lz - Xt / Zt);
+            }
+            if (seg == 0) p.row_ent[row] = ent;
+          }
+          lse_s[r] = lse2;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+      }
+      // This thread owns key (tile * 128 + quarter * 32 + lane).  Rows: for W <= 64 the block's
+      // rows [sub * 64, sub * 64 + 64) of every tile (two heads at W = 32, one at W = 64); for
+      // W = 128 the 128 rows of head (sub & 1) on every other tile, tiles alternating between the
+      // warps with sub >> 1 = 0 and 1, so that a head's column sum never spans two warps.
+      constexpr int kChunks = (W == 128) ? 4 : 2;
+      const int col0 = (W == 128) ? (sub & 1) * 128 : sub * 64;   // first accumulator column = local row
+      const float inv_w = 1.0f / (float)p.window;
+      const int row0 = rb * kRowBlock + col0;                // first score row (within the group) of this thread
+      const bool warp_active = col0 < rows_here;
+      const int h0 = g * p.group + row0 / p.window;          // (first) head of this thread
+      // sum over the chunk's 32 rows of 2^(x - lse) for this thread's key, all rows visible
+      auto colsum = [&](int c) {
+        const float4* l4 = reinterpret_cast<const float4*>(lse_s + col0 + c * 32);
+        float s = 0.f;
+#pragma unroll
+        for (int e4 = 0; e4 < 8; ++e4) {
+          const float4 l = l4[e4];
+          const float ls[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int e = 4 * e4 + q;
+            const float x = fmaf(v[e], p.c2, -ls[q]);
+            s += ((e & 7) < kPoly2) ? exp2_poly(fmaxf(x, -125.f)) : fast_exp2(x);
           }
         }
-        tc_fence_before();
-        mbar_arrive(bars + 8 * (kBarAccEmpty + a));
-        if (half_active && j < p.n_keys) {
+        return s;
+      };
+      // same for a tile that holds window keys: window row i sees key j only if i >= i_min
+      auto colsum_masked = [&](int c, int i_min) {
+        float s = 0.f;
 #pragma unroll
-          for (int hh = 0; hh < kHeads; ++hh) {
-            const int lr = row0 + hh * (128 / kHeads);       // first local row of this head slice
-            if (lr < p.rows_pg) {
-              const int h = g * p.group + lr / p.window;
-              p.cols[(size_t)h * p.col_stride + j] = acc[hh] * inv_w;
-            }
+        for (int e = 0; e < 32; ++e) {
+          const int i = (row0 + c * 32 + e) % p.window;
+          const float x = fmaf(v[e], p.c2, -lse_s[col0 + c * 32 + e]);
+          s += (i >= i_min) ? fast_exp2(x) : 0.f;
+        }
+        return s;
+      };
+      for (int t = 0; t < n_my; ++t) {
+        if (!acc_full(t)) break;
+        const int tile = tile_of(t);
+        const int j = tile * kKeyTile + quarter * 32 + lane;
+        const bool plain = tile < first_tail_tile;
+        const int i_min = j - (p.n_keys - p.window);        // window rows i < i_min do not see key j
+        const uint32_t taddr = tmem + lane_base + (uint32_t)((t % kAccStages) * 256 + col0);
+        const bool mine = warp_active && (W != 128 || (t & 1) == (sub >> 1));
+        float sc[kChunks];
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          sc[c] = 0.f;
+          if (mine) {
+            tmem_ld32(taddr + c * 32, v);
+            tmem_ld_wait(v);
+          }
+          if (c == kChunks - 1) acc_release(t);             // every load of the tile has landed
+          if (mine) sc[c] = plain ? colsum(c) : colsum_masked(c, i_min);
+        }
+        if (mine && j < p.n_keys) {
+          if (W == 32) {
+            p.cols[(size_t)h0 * p.col_stride + j] = sc[0] * inv_w;
+            if (row0 + 32 < p.rows_pg) p.cols[(size_t)(h0 + 1) * p.col_stride + j] = sc[1] * inv_w;
+          } else {
+            float tot = 0.f;
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c) tot += sc[c];
+            p.cols[(size_t)h0 * p.col_stride + j] = tot * inv_w;
           }
         }
       }
     }
+    tmem_ld_wait();
   }
 
   // ---------------- teardown ----------------
@@ -515,15 +607,15 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   int segs = ctx.sm_count / units;
   if (segs < 1) segs = 1;
   if (segs > p.n_tiles) segs = p.n_tiles;
-  if (segs > kMaxParts) segs = kMaxParts;
+  if (2 * segs > kMaxParts) segs = kMaxParts / 2;   // pass 1 leaves two partial statistics per segment
   p.segs = segs;
   p.c2 = a.scale * kLog2e;
   p.row_part = ctx.ws.row_part;
-  p.row_lse2 = ctx.ws.row_lse2;
+  p.row_ent = ctx.ws.row_ent;
   p.cols = a.cols;
   p.col_stride = a.col_stride;
   p.status = ctx.ws.status;
-  *parts_out = segs;
+  *parts_out = 2 * segs;
   const int grid = units * segs;
   const int d = ctx.cfg.head_dim, w = ctx.cfg.window;
   if (d == 128) return pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);
