@@ -128,26 +128,60 @@ __device__ __forceinline__ void tmem_ld_wait(float (&v)[32]) {
       :: "memory");
 }
 
-// 2^x on the FMA pipe for x in [-125, 126]: round-to-nearest split x = n + f with the
+// Two fp32 values in one 64-bit register, for the packed fp32 instructions of sm_100
+// (one issue slot for two results).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t r, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 2^x for a pair, on the FMA pipe, x in [-125, 126]: round-to-nearest split x = n + f with the
 // 1.5 * 2^23 trick (n lands in the low mantissa bits of t), a degree-3 minimax polynomial
 // for 2^f on [-0.5, 0.5] (relative error 7.5e-5), and n added into the exponent field.
-__device__ __forceinline__ float exp2_poly(float x) {
-  const float t = x + 12582912.0f;
-  const float f = x - (t - 12582912.0f);
-  float p = fmaf(0.0551716685f, f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x) {
+  const uint64_t magic = pack2(12582912.0f, 12582912.0f);
+  const uint64_t t = add2(x, magic);
+  const uint64_t f = sub2(x, sub2(t, magic));
+  uint64_t p = fma2(pack2(0.0551716685f, 0.0551716685f), f, pack2(0.2426111251f, 0.2426111251f));
+  p = fma2(p, f, pack2(0.6932609677f, 0.6932609677f));
+  p = fma2(p, f, pack2(0.9999280572f, 0.9999280572f));
+  float t0, t1, p0, p1;
+  unpack2(t, t0, t1);
+  unpack2(p, p0, p1);
+  return pack2(__int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23)),
+               __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23)));
 }
-// Of every 8 consecutive elements the first kPoly1 (pass 1) / kPoly2 (pass 2) take the
-// polynomial, the rest the special-function unit.
-#ifndef SKV_POLY1
-#define SKV_POLY1 0
-#endif
+// 2^x for a pair on the special-function unit.
+__device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
+  float x0, x1;
+  unpack2(x, x0, x1);
+  return pack2(fast_exp2(x0), fast_exp2(x1));
+}
+// In pass 2, of every 8 consecutive element pairs the first kPoly2 take the polynomial, the
+// rest the special-function unit: the two pipes work side by side (2 of 8 measured best).
 #ifndef SKV_POLY2
-#define SKV_POLY2 0
+#define SKV_POLY2 2
 #endif
-constexpr int kPoly1 = SKV_POLY1, kPoly2 = SKV_POLY2;
+constexpr int kPoly2 = SKV_POLY2;
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, 8-row
 // groups 1024 bytes apart (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).
@@ -174,7 +208,8 @@ struct Smem {
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kQBytes;
   static constexpr int kLseOff = kKOff + kStages * kKBytes;          // 256 floats
-  static constexpr int kBarOff = kLseOff + kRowBlock * 4;
+  static constexpr int kMergeOff = kLseOff + kRowBlock * 4;          // 256 x (M, Z, X) for the pass-2 merge
+  static constexpr int kBarOff = kMergeOff + kRowBlock * 16;
   static constexpr int kBytes = kBarOff + 256;
   static constexpr int kAlloc = kBytes + 1024;             // slack to align the base to 1024 bytes
 };
@@ -327,12 +362,13 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       const int i_win = (rb * kRowBlock + row_in_block) % p.window;      // window row index of this score row
       const int t_pos = p.n_keys - p.window + i_win;                     // its position: sees keys <= t_pos
       float ref = -INFINITY, Z = 0.f, U = 0.f;
-      // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible
+      // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible.
+      // (Scalar arithmetic: here the packed form measured slower, the pairs are unpacked twice.)
       auto accumulate = [&]() {
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const float x = fmaf(v[e], p.c2, -ref);
-          const float pr = ((e & 7) < kPoly1) ? exp2_poly(fminf(fmaxf(x, -125.f), 126.f)) : fast_exp2(x);
+          const float pr = fast_exp2(x);
           Z += pr;
           U = fmaf(pr, x, U);
         }
@@ -393,40 +429,65 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         p.row_part[(size_t)(seg * 2 + ch) * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
             n_my > 0 ? make_float4(ref, Z, U, 0.f) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
     } else {
-      // pass 2.  First the compute threads merge the partial statistics of this block's rows:
-      // with l_s = ref_s + log2 Z_s (a partial's log-sum-exp) and M = max_s l_s,
-      //   lse2 = M + log2 sum_s 2^(l_s - M),
-      //   entropy = ln2 (lse2 - M - sum_s 2^(l_s - M) (ref_s - M + U_s / Z_s) / sum_s 2^(l_s - M)).
-      // Padded rows get +inf so that they contribute 2^(-inf) = 0.
+      // pass 2.  First the compute threads merge the partial statistics of this block's rows,
+      // two threads per row (each takes every other partial, loads batched), then one of them
+      // folds the two.  With l_s = ref_s + log2 Z_s (a partial's log-sum-exp), a running maximum
+      // M, Zt = sum_s 2^(l_s - M) and Xt = sum_s 2^(l_s - M) (ref_s - M + U_s / Z_s):
+      //   lse2 = M + log2 Zt,   entropy = ln2 (log2 Zt - Xt / Zt)                (Eq. 4, one row)
+      // lse_s holds -lse2; padded rows get -inf so that they contribute 2^(-inf) = 0.
       {
-        const int r = (int)threadIdx.x - 64;
-        if (r < kRowBlock) {
-          float lse2 = INFINITY, ent = 0.f;
-          const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
-          const int parts = 2 * p.segs;
-          if (r < rows_here) {
-            float M = -INFINITY;
-            for (int s = 0; s < parts; ++s) {
-              const float4 pv = p.row_part[(size_t)s * p.rows_pad + row];
-              if (pv.y > 0.f) M = fmaxf(M, pv.x + log2f(pv.y));
-            }
+        const int ct = (int)threadIdx.x - 64;
+        const int r = ct & (kRowBlock - 1), hp = ct >> 8;
+        const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
+        const int parts = 2 * p.segs;
+        float M = -INFINITY, Zt = 0.f, Xt = 0.f;
+        auto fold = [&](float ref_s, float Z_s, float X_s) {     // X_s = sum 2^(..)(.. - ref_s), relative to ref_s
+          if (!(Z_s > 0.f)) return;
+          const float l = ref_s + log2f(Z_s);
+          if (l > M) {
             if (M != -INFINITY) {
-              float Zt = 0.f, Xt = 0.f;
-              for (int s = 0; s < parts; ++s) {
-                const float4 pv = p.row_part[(size_t)s * p.rows_pad + row];
-                if (pv.y > 0.f) {
-                  const float wgt = fast_exp2(pv.x + log2f(pv.y) - M);
-                  Zt += wgt;
-                  Xt = fmaf(wgt, (pv.x - M) + pv.z / pv.y, Xt);
-                }
-              }
-              const float lz = log2f(Zt);
-              lse2 = M + lz;
-              ent = kLn2 * (lz - Xt / Zt);
+              const float d = M - l, f = fast_exp2(d);
+              Xt = f * fmaf(d, Zt, Xt);
+              Zt = f * Zt;
             }
-            if (seg == 0) p.row_ent[row] = ent;
+            M = l;
           }
-          lse_s[r] = lse2;
+          const float wgt = fast_exp2(l - M);
+          Zt += wgt;
+          Xt = fmaf(wgt, (ref_s - M) + X_s / Z_s, Xt);
+        };
+        if (r < rows_here) {
+          constexpr int kBatch = 6;
+          for (int s0 = hp; s0 < parts; s0 += 2 * kBatch) {
+            float4 pv[kBatch];
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+              const int sidx = s0 + 2 * b;
+              pv[b] = sidx < parts ? __ldg(&p.row_part[(size_t)sidx * p.rows_pad + row])
+                                   : make_float4(-INFINITY, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) fold(pv[b].x, pv[b].y, pv[b].z);
+          }
+        }
+        float4* merge_s = reinterpret_cast<float4*>(sm + L::kMergeOff);
+        if (hp == 1) merge_s[r] = make_float4(M, Zt, Xt, 0.f);
+        asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+        if (hp == 0) {
+          // the other thread's result is one more partial: (reference M', sum Zt', Xt' relative to M')
+          const float4 o = merge_s[r];
+          if (o.y > 0.f) {
+            // its log-sum-exp is M' + log2 Zt'; fold() expects (ref, Z, X) with X relative to ref
+            fold(o.x, o.y, o.z);
+          }
+          float nlse = -INFINITY, ent = 0.f;
+          if (r < rows_here && Zt > 0.f) {
+            const float lz = log2f(Zt);
+            nlse = -(M + lz);
+            ent = kLn2 * (lz - Xt / Zt);
+          }
+          if (r < rows_here && seg == 0) p.row_ent[row] = ent;
+          lse_s[r] = nlse;
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
       }
@@ -441,21 +502,32 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       const bool warp_active = col0 < rows_here;
       const int h0 = g * p.group + row0 / p.window;          // (first) head of this thread
       // sum over the chunk's 32 rows of 2^(x - lse) for this thread's key, all rows visible
+      // (packed arithmetic; lse_s holds -lse)
       auto colsum = [&](int c) {
-        const float4* l4 = reinterpret_cast<const float4*>(lse_s + col0 + c * 32);
-        float s = 0.f;
+        const ulonglong2* l2 = reinterpret_cast<const ulonglong2*>(lse_s + col0 + c * 32);
+        const uint64_t c22 = pack2(p.c2, p.c2);
+        uint64_t s2 = pack2(0.f, 0.f);
 #pragma unroll
         for (int e4 = 0; e4 < 8; ++e4) {
-          const float4 l = l4[e4];
-          const float ls[4] = {l.x, l.y, l.z, l.w};
+          const ulonglong2 l = l2[e4];                      // -lse of rows 4 e4 .. 4 e4 + 3
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int e = 4 * e4 + q;
-            const float x = fmaf(v[e], p.c2, -ls[q]);
-            s += ((e & 7) < kPoly2) ? exp2_poly(fmaxf(x, -125.f)) : fast_exp2(x);
+          for (int q = 0; q < 2; ++q) {
+            const int pr = 2 * e4 + q;
+            const uint64_t x2 = fma2(pack2(v[2 * pr], v[2 * pr + 1]), c22, q == 0 ? l.x : l.y);
+            uint64_t p2;
+            if ((pr & 7) < kPoly2) {
+              float x0, x1;
+              unpack2(x2, x0, x1);
+              p2 = exp2_poly2(pack2(fminf(fmaxf(x0, -125.f), 126.f), fminf(fmaxf(x1, -125.f), 126.f)));
+            } else {
+              p2 = exp2_sfu2(x2);
+            }
+            s2 = add2(s2, p2);
           }
         }
-        return s;
+        float a, b;
+        unpack2(s2, a, b);
+        return a + b;
       };
       // same for a tile that holds window keys: window row i sees key j only if i >= i_min
       auto colsum_masked = [&](int c, int i_min) {
@@ -463,7 +535,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const int i = (row0 + c * 32 + e) % p.window;
-          const float x = fmaf(v[e], p.c2, -lse_s[col0 + c * 32 + e]);
+          const float x = fmaf(v[e], p.c2, lse_s[col0 + c * 32 + e]);
           s += (i >= i_min) ? fast_exp2(x) : 0.f;
         }
         return s;
