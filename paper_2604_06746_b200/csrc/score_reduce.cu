@@ -94,52 +94,89 @@ __global__ void reduce_columns(const float* __restrict__ cols, long long col_str
 constexpr int kHsCluster = 8;
 constexpr int kHsThreads = 1024;
 constexpr int kHsBins = 2048;
+constexpr int kHsCopies = 8;      // each bin is kept 8 times (lane & 7) so that a warp's hits on one bin spread
+constexpr int kHsItems = 16;      // entries per thread kept in registers between the sweeps
 
+// Shared memory of head_stats: hist[kHsBins][kHsCopies] | merged[kHsBins] (dynamic, 72 KB).
 __global__ void __cluster_dims__(kHsCluster, 1, 1) __launch_bounds__(kHsThreads)
 head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rho,
            float* __restrict__ head_part) {
-  __shared__ unsigned hist[kHsBins];         // this CTA's counts
-  __shared__ unsigned merged[kHsBins];       // cluster-wide counts (CTA 0's copy is the one used)
+  extern __shared__ unsigned hs_smem[];
+  unsigned* hist = hs_smem;                          // this CTA's counts, kHsCopies per bin
+  unsigned* merged = hs_smem + kHsBins * kHsCopies;  // cluster-wide counts (CTA 0's copy is the one used)
   __shared__ float red[33];
-  __shared__ float slots[2 * kHsCluster];    // CTA 0: per-CTA {sum of squares, mass above}
+  __shared__ float slots[2 * kHsCluster];            // CTA 0: per-CTA {sum of squares, mass above}
   __shared__ unsigned sel_bin, sel_rem;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int head = blockIdx.x / kHsCluster;
   const float* a = cols + (size_t)head * col_stride;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, copy = tid & (kHsCopies - 1);
   const int per = (n + kHsCluster - 1) / kHsCluster;
   const int lo = rank * per, hi = min(n, lo + per);
+  const bool in_regs = per <= kHsItems * kHsThreads;  // otherwise the second sweep reads memory again
   unsigned* merged0 = cluster.map_shared_rank(merged, 0);
 
-  for (int b = tid; b < kHsBins; b += kHsThreads) { hist[b] = 0; merged[b] = 0; }
+  auto clear = [&]() {
+    for (int b = tid; b < kHsBins * kHsCopies; b += kHsThreads) hist[b] = 0;
+    for (int b = tid; b < kHsBins; b += kHsThreads) merged[b] = 0;
+  };
+  auto push = [&]() {                                // this CTA's counts into CTA 0's merged[]
+    for (int b = tid; b < kHsBins; b += kHsThreads) {
+      unsigned c = 0;
+#pragma unroll
+      for (int k = 0; k < kHsCopies; ++k) c += hist[b * kHsCopies + k];
+      if (c) atomicAdd(&merged0[b], c);
+    }
+  };
+
+  clear();
+  float reg[kHsItems];
+#pragma unroll
+  for (int e = 0; e < kHsItems; ++e) {
+    const int j = lo + e * kHsThreads + tid;
+    reg[e] = (in_regs && j < hi) ? a[j] : -1.f;      // -1 marks "no entry" (real entries are >= 0)
+  }
   cluster.sync();
   float sq = 0.f;
-  for (int j = lo + tid; j < hi; j += kHsThreads) {
-    const float v = a[j];
-    sq = fmaf(v, v, sq);
-    atomicAdd(&hist[(__float_as_uint(v) >> 20) & 0x7ffu], 1u);
+  if (in_regs) {
+#pragma unroll
+    for (int e = 0; e < kHsItems; ++e)
+      if (reg[e] >= 0.f) {
+        sq = fmaf(reg[e], reg[e], sq);
+        atomicAdd(&hist[((__float_as_uint(reg[e]) >> 20) & 0x7ffu) * kHsCopies + copy], 1u);
+      }
+  } else {
+    for (int j = lo + tid; j < hi; j += kHsThreads) {
+      const float v = a[j];
+      sq = fmaf(v, v, sq);
+      atomicAdd(&hist[((__float_as_uint(v) >> 20) & 0x7ffu) * kHsCopies + copy], 1u);
+    }
   }
   __syncthreads();
-  for (int b = tid; b < kHsBins; b += kHsThreads)
-    if (hist[b]) atomicAdd(&merged0[b], hist[b]);
+  push();
   cluster.sync();
   if (tid < 32) radix_pick_from_top(merged0, kHsBins, (unsigned)k_rho, &sel_bin, &sel_rem);
   __syncthreads();
   const unsigned b1 = sel_bin, rem1 = sel_rem;
   cluster.sync();                            // every CTA has read the level-1 counts
-  for (int b = tid; b < kHsBins; b += kHsThreads) { hist[b] = 0; merged[b] = 0; }
+  clear();
   cluster.sync();
   float mass = 0.f;
-  for (int j = lo + tid; j < hi; j += kHsThreads) {
-    const float v = a[j];
+  auto second = [&](float v) {
     const unsigned u = __float_as_uint(v), top = (u >> 20) & 0x7ffu;
     if (top > b1) mass += v;
-    else if (top == b1) atomicAdd(&hist[(u >> 9) & 0x7ffu], 1u);
+    else if (top == b1) atomicAdd(&hist[((u >> 9) & 0x7ffu) * kHsCopies + copy], 1u);
+  };
+  if (in_regs) {
+#pragma unroll
+    for (int e = 0; e < kHsItems; ++e)
+      if (reg[e] >= 0.f) second(reg[e]);
+  } else {
+    for (int j = lo + tid; j < hi; j += kHsThreads) second(a[j]);
   }
   __syncthreads();
-  for (int b = tid; b < kHsBins; b += kHsThreads)
-    if (hist[b]) atomicAdd(&merged0[b], hist[b]);
+  push();
   const float tot_sq = block_sum_1024(sq, red);
   const float tot_mass = block_sum_1024(mass, red);
   if (tid == 0) {
@@ -231,9 +268,12 @@ cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stri
   if (with_head_stats) {
     int k_rho = n / 10;
     if (k_rho < 1) k_rho = 1;
-    head_stats<<<ctx.cfg.n_q_heads * kHsCluster, kHsThreads, 0, st>>>(cols, col_stride, n, k_rho,
-                                                                      ctx.ws.head_part);
-    const cudaError_t e = cudaGetLastError();
+    const int smem = (kHsBins * kHsCopies + kHsBins) * (int)sizeof(unsigned);
+    cudaError_t e = cudaFuncSetAttribute(head_stats, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    head_stats<<<ctx.cfg.n_q_heads * kHsCluster, kHsThreads, smem, st>>>(cols, col_stride, n, k_rho,
+                                                                         ctx.ws.head_part);
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
