@@ -156,7 +156,11 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   __syncthreads();
   push();
   cluster.sync();
-  if (tid < 32) radix_pick_from_top(merged0, kHsBins, (unsigned)k_rho, &sel_bin, &sel_rem);
+  // copy the cluster-wide counts into this CTA (all threads, remote reads in parallel), then pick
+  if (rank != 0)
+    for (int b = tid; b < kHsBins; b += kHsThreads) merged[b] = merged0[b];
+  __syncthreads();
+  if (tid < 32) radix_pick_from_top(merged, kHsBins, (unsigned)k_rho, &sel_bin, &sel_rem);
   __syncthreads();
   const unsigned b1 = sel_bin, rem1 = sel_rem;
   cluster.sync();                            // every CTA has read the level-1 counts

@@ -20,6 +20,7 @@ constexpr int kSelThreads = 1024;
 constexpr int kSelBins = 2048;
 constexpr int kSelCopies = 8;
 constexpr int kSelItems = 4;     // consecutive elements per thread in the output sweep
+constexpr int kSelBatch = 8;     // loads in flight per thread in the counting sweeps
 
 // Larger float -> larger unsigned; -0 is folded onto +0.
 __device__ __forceinline__ unsigned order_key(float v) {
@@ -66,10 +67,19 @@ select_topk(const float* __restrict__ scores, long long row_stride, int n, int b
       for (int b = tid; b < kSelBins; b += kSelThreads) merged[b] = 0;
       cluster.sync();
       const unsigned bmask = (1u << widths[pass]) - 1u;
-      for (int j = lo + tid; j < hi; j += kSelThreads) {
-        const unsigned u = order_key(s[j]);
-        if ((u & prefix_mask) == prefix)
-          atomicAdd(&hist[((u >> shifts[pass]) & bmask) * kSelCopies + copy], 1u);
+      for (int j0 = lo + tid; j0 < hi; j0 += kSelThreads * kSelBatch) {
+        float val[kSelBatch];
+#pragma unroll
+        for (int e = 0; e < kSelBatch; ++e) {
+          const int j = j0 + e * kSelThreads;
+          val[e] = j < hi ? s[j] : 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < kSelBatch; ++e) {
+          const unsigned u = order_key(val[e]);
+          if (j0 + e * kSelThreads < hi && (u & prefix_mask) == prefix)
+            atomicAdd(&hist[((u >> shifts[pass]) & bmask) * kSelCopies + copy], 1u);
+        }
       }
       __syncthreads();
       for (int b = tid; b < kSelBins; b += kSelThreads) {
@@ -79,7 +89,11 @@ select_topk(const float* __restrict__ scores, long long row_stride, int n, int b
         if (c) atomicAdd(&merged0[b], c);
       }
       cluster.sync();
-      if (tid < 32) radix_pick_from_top(merged0, 1 << widths[pass], remaining, &sel_bin, &sel_rem);
+      // copy the cluster-wide counts into this CTA (remote reads in parallel), then pick locally
+      if (rank != 0)
+        for (int b = tid; b < kSelBins; b += kSelThreads) merged[b] = merged0[b];
+      __syncthreads();
+      if (tid < 32) radix_pick_from_top(merged, 1 << widths[pass], remaining, &sel_bin, &sel_rem);
       __syncthreads();
       prefix |= sel_bin << shifts[pass];
       prefix_mask |= bmask << shifts[pass];
@@ -92,10 +106,20 @@ select_topk(const float* __restrict__ scores, long long row_stride, int n, int b
 
   // keys greater than / equal to the threshold in this CTA's slice -> offsets of the slice
   unsigned my_gt = 0, my_eq = 0;
-  for (int j = lo + tid; j < hi; j += kSelThreads) {
-    const unsigned u = order_key(s[j]);
-    my_gt += (keep_all || u > thr) ? 1u : 0u;
-    my_eq += (!keep_all && u == thr) ? 1u : 0u;
+  for (int j0 = lo + tid; j0 < hi; j0 += kSelThreads * kSelBatch) {
+    float val[kSelBatch];
+#pragma unroll
+    for (int e = 0; e < kSelBatch; ++e) {
+      const int j = j0 + e * kSelThreads;
+      val[e] = j < hi ? s[j] : 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < kSelBatch; ++e) {
+      const unsigned u = order_key(val[e]);
+      const bool in = j0 + e * kSelThreads < hi;
+      my_gt += (in && (keep_all || u > thr)) ? 1u : 0u;
+      my_eq += (in && !keep_all && u == thr) ? 1u : 0u;
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
