@@ -34,6 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant
 # kernel, from the ncu capture summarised under profiles/; None until a capture exists.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_NOTE = None
 
 
 def load_peaks():
@@ -58,7 +59,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -113,6 +114,60 @@ def cpu_baseline(wl, pl, kv_budget, n_layers_sample=1):
                       f"K/V), {per_layer:.2f} s per layer, scaled to all layers"}
 
 
+def measure_e2e(wl, pf, layers, hidden, positions, dev, steps, world):
+    """The same step with HOST buffers: every step copies each layer's q / K / V, the hidden states
+    and the position ids from pinned host memory to the device, runs the path through the C ABI,
+    and copies the results (compacted K / V, gathered hidden states and positions, both index sets,
+    the metric table) back to pinned host memory.  One stream, copies inside the timed region."""
+    host_layers = []
+    try:
+        for t in layers:
+            host_layers.append({k: torch.empty(t[k].shape, dtype=t[k].dtype, pin_memory=True).copy_(t[k])
+                                for k in ("q_win", "k", "v")})
+        host_hidden = torch.empty(hidden.shape, dtype=hidden.dtype, pin_memory=True).copy_(hidden)
+        host_pos = torch.empty(positions.shape, dtype=positions.dtype, pin_memory=True).copy_(positions)
+        outs = {"k_out": pf.k_out, "v_out": pf.v_out, "hidden_out": pf.hidden_out, "pos_out": pf.pos_out,
+                "i_kv": pf.i_kv, "i_struct": pf.i_struct, "metrics": pf.metrics}
+        host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
+    except RuntimeError as e:
+        return {"value": None, "unit": UNIT, "unavailable": f"pinned host allocation failed: {e}"[:200]}
+    h2d = sum(sum(t[k].numel() * t[k].element_size() for k in t) for t in host_layers) \
+        + host_hidden.numel() * host_hidden.element_size() + host_pos.numel() * host_pos.element_size()
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+
+    def step():
+        for l, (hd, t) in enumerate(zip(host_layers, layers)):
+            for k in ("q_win", "k", "v"):
+                t[k].copy_(hd[k], non_blocking=True)
+            pf.score(l, t["q_win"], t["k"], t["scale"])
+        hidden.copy_(host_hidden, non_blocking=True)
+        positions.copy_(host_pos, non_blocking=True)
+        pf.detect_and_select(len(layers))
+        for l, t in enumerate(layers):
+            pf.compact_kv(l, t["k"], t["v"])
+        pf.compact_hidden(hidden, positions)
+        for k, v in outs.items():
+            host_out[k].copy_(v, non_blocking=True)
+
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    if world > 1:
+        import torch.distributed as dist
+        tms = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ms = float(tms.item())
+    return {"value": world * wl.seq / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "note": "inputs in pinned host memory, copied every step; results copied back to pinned host memory"}
+
+
 def run_reference(args):
     """The reference arm of this build is the CPU oracle (the paper ships no code)."""
     from paper_2604_06746_b200 import synth
@@ -148,13 +203,16 @@ def workload_config(wl, kv_budget):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama128k")
     ap.add_argument("--budget", type=int, default=16384)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="profile a prefix of the layers (0 = all)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -172,6 +230,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     wl = synth.WORKLOADS[args.workload]
+    if args.layers:
+        wl = wl.scaled(wl.seq, n_layers=args.layers, name=f"{wl.name}[first {args.layers} layers]",
+                       budgets=wl.budgets)
     pl = synth.plan(wl)
     kv_budget = args.budget or wl.budget
     st_budget = wl.struct_budget(kv_budget)
@@ -229,6 +290,8 @@ def main():
         tms = torch.tensor([ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tms, op=dist.ReduceOp.MAX)
         ms = float(tms.item())
+    e2e = None if args.no_e2e else measure_e2e(wl, pf, layers, hidden, positions, dev, args.e2e_steps, world)
+    assert pf.ctx.poll_device_status() == binding.OK
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -250,6 +313,7 @@ def main():
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH
+    roof["traffic_note"] = NCU_TRAFFIC_NOTE
     roof["kernel"] = "structkv_score_layer (both scorer passes + reductions), per layer"
     roof["us_per_layer"] = score_s * 1e6
     roof["peaks"] = peaks["source"]
@@ -259,14 +323,14 @@ def main():
     compaction = {"achieved": comp_bytes / comp_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                   "frac": comp_bytes / comp_s / 1e9 / peaks["hbm_gbs"], "bytes_per_step": comp_bytes}
 
-    n_launch = L * (5 if not (args.flags & binding.FLAG_NO_HEAD_STATS) else 5) + 1 + 2 + 2 * L + 2
+    n_launch = L * (5 if not (args.flags & binding.FLAG_NO_HEAD_STATS) else 4) + 1 + 2 + 2 * L + 2
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32",
             "data": "synthetic", "config": workload_config(wl, kv_budget), "pivot": pf.pivot,
             "phase_ms_per_step": {k: v / args.steps for k, v in phase_ms.items()},
             "roofline": roof, "compaction": compaction, "clocks": clocks,
-            "gpu_launches": n_launch * args.steps, "e2e": None}
+            "gpu_launches": n_launch * args.steps, "e2e": e2e}
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, pl, kv_budget, n_layers_sample=1)
     print(json.dumps(line))
