@@ -33,8 +33,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant
 # kernel, from the ncu capture summarised under profiles/; None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
-NCU_TRAFFIC_NOTE = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 557.0e6
+NCU_TRAFFIC_NOTE = ("dram read+write of the two tc_score launches of one layer (llama128k shape), "
+                    "profiles/tc_score_llama128k_ncu_full.md; valid for the llama128k workload only")
 
 
 def load_peaks():
@@ -312,7 +313,7 @@ def main():
         roof = {"bound": "tensor", "achieved": flops / score_s / 1e12, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH
+    roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH if wl.name.startswith("llama128k") else None
     roof["traffic_note"] = NCU_TRAFFIC_NOTE
     roof["kernel"] = "structkv_score_layer (both scorer passes + reductions), per layer"
     roof["us_per_layer"] = score_s * 1e6
