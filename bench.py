@@ -124,10 +124,10 @@ def measure_e2e(wl, pf, layers, hidden, positions, dev, steps, world):
     try:
         for t in layers:
             host_layers.append({k: torch.empty(t[k].shape, dtype=t[k].dtype, pin_memory=True).copy_(t[k])
-                                for k in ("q_win", "k", "v")})
+                                for k in ("q_win", "kv")})
         host_hidden = torch.empty(hidden.shape, dtype=hidden.dtype, pin_memory=True).copy_(hidden)
         host_pos = torch.empty(positions.shape, dtype=positions.dtype, pin_memory=True).copy_(positions)
-        outs = {"k_out": pf.k_out, "v_out": pf.v_out, "hidden_out": pf.hidden_out, "pos_out": pf.pos_out,
+        outs = {"kv_out": pf.kv_out, "hidden_out": pf.hidden_out, "pos_out": pf.pos_out,
                 "i_kv": pf.i_kv, "i_struct": pf.i_struct, "metrics": pf.metrics}
         host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
     except RuntimeError as e:
@@ -138,14 +138,14 @@ def measure_e2e(wl, pf, layers, hidden, positions, dev, steps, world):
 
     def step():
         for l, (hd, t) in enumerate(zip(host_layers, layers)):
-            for k in ("q_win", "k", "v"):
+            for k in ("q_win", "kv"):
                 t[k].copy_(hd[k], non_blocking=True)
             pf.score(l, t["q_win"], t["k"], t["scale"])
         hidden.copy_(host_hidden, non_blocking=True)
         positions.copy_(host_pos, non_blocking=True)
         pf.detect_and_select(len(layers))
         for l, t in enumerate(layers):
-            pf.compact_kv(l, t["k"], t["v"])
+            pf.compact_kv(l, t["k"], t["v"], t.get("kv"))
         pf.compact_hidden(hidden, positions)
         for k, v in outs.items():
             host_out[k].copy_(v, non_blocking=True)
@@ -259,7 +259,7 @@ def main():
         pf.detect_and_select(len(layers))
         if timed: e[2].record()
         for l, t in enumerate(layers):
-            pf.compact_kv(l, t["k"], t["v"])
+            pf.compact_kv(l, t["k"], t["v"], t.get("kv"))
         pf.compact_hidden(hidden, positions)
         if timed: e[3].record()
         return e
@@ -324,7 +324,7 @@ def main():
     compaction = {"achieved": comp_bytes / comp_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                   "frac": comp_bytes / comp_s / 1e9 / peaks["hbm_gbs"], "bytes_per_step": comp_bytes}
 
-    n_launch = L * (5 if not (args.flags & binding.FLAG_NO_HEAD_STATS) else 4) + 1 + 2 + 2 * L + 2
+    n_launch = L * (5 if not (args.flags & binding.FLAG_NO_HEAD_STATS) else 4) + 1 + 2 + L + 2
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32",

@@ -1,13 +1,39 @@
 // Row gather / compaction: dst[s, r, :] = src[s, idx[r], :], byte exact.  Rows are split into
 // 16-byte (or 4-byte / 1-byte) units; consecutive threads take consecutive units of a row, so
-// writes are fully coalesced and reads are coalesced within each gathered row.
+// writes are fully coalesced and reads are coalesced within each gathered row.  Two loads in
+// flight per thread and up to 64 resident blocks per SM measured best on B200 (more unrolling
+// or fewer, fatter blocks lose 10-25 % of the copy bandwidth).
 #include "common.cuh"
 
 namespace skv {
 namespace {
 
-constexpr int kCpThreads = 256;
-constexpr int kCpUnroll = 4;
+#ifndef SKV_CP_THREADS
+#define SKV_CP_THREADS 256
+#endif
+#ifndef SKV_CP_UNROLL
+#define SKV_CP_UNROLL 2
+#endif
+#ifndef SKV_CP_BLOCKS_PER_SM
+#define SKV_CP_BLOCKS_PER_SM 64
+#endif
+constexpr int kCpThreads = SKV_CP_THREADS;
+constexpr int kCpUnroll = SKV_CP_UNROLL;
+
+// Rows are read once and written once: loads bypass L1 allocation, stores are streaming.
+template <typename V> __device__ __forceinline__ V ld_stream(const V* p) { return *p; }
+template <typename V> __device__ __forceinline__ void st_stream(V* p, const V& v) { *p = v; }
+#ifndef SKV_CP_PLAIN
+template <> __device__ __forceinline__ uint4 ld_stream<uint4>(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+template <> __device__ __forceinline__ void st_stream<uint4>(uint4* p, const uint4& v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+#endif
 
 template <typename V>
 __global__ void __launch_bounds__(kCpThreads)
@@ -30,8 +56,8 @@ gather_rows(const char* __restrict__ src, long long slab_stride, long long row_s
         const int s = (int)(row / n_idx), r = (int)(row - (long long)s * n_idx);
         const int j = __ldg(idx + r);
         if (j >= 0 && j < n_rows_src) {
-          val[e] = *reinterpret_cast<const V*>(src + s * slab_stride + j * row_stride +
-                                               (long long)c * sizeof(V));
+          val[e] = ld_stream(reinterpret_cast<const V*>(src + s * slab_stride + j * row_stride +
+                                                        (long long)c * sizeof(V)));
           ok[e] = true;
         } else if (c == 0) {
           atomicCAS(status, 0, (int)STRUCTKV_ERR_INVALID_ARG);
@@ -41,7 +67,7 @@ gather_rows(const char* __restrict__ src, long long slab_stride, long long row_s
 #pragma unroll
     for (int e = 0; e < kCpUnroll; ++e) {
       const long long u = u0 + e * stride;
-      if (ok[e]) *reinterpret_cast<V*>(dst + u * (long long)sizeof(V)) = val[e];
+      if (ok[e]) st_stream(reinterpret_cast<V*>(dst + u * (long long)sizeof(V)), val[e]);
     }
   }
 }
@@ -60,7 +86,7 @@ cudaError_t launch_compact(const void* src, long long slab_stride, long long row
   const int upr = row_bytes / unit;
   const long long total = (long long)n_slabs * n_idx * upr;
   long long blocks = (total + (long long)kCpThreads * kCpUnroll - 1) / ((long long)kCpThreads * kCpUnroll);
-  const long long cap = (long long)sm_count * 16;
+  const long long cap = (long long)sm_count * SKV_CP_BLOCKS_PER_SM;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   const char* s = (const char*)src;

@@ -37,8 +37,11 @@ class Prefill:
         self.i_struct = torch.zeros((struct_budget,), dtype=i32, device=dev)
         n_kv_out = n_layers if keep_kv else 1
         self.keep_kv = keep_kv
-        self.k_out = torch.empty((n_kv_out, n_kv_heads, kv_budget, head_dim), dtype=dtype, device=dev)
-        self.v_out = torch.empty_like(self.k_out)
+        # compacted K and V of a layer sit in one allocation [2, H_kv, B, d]: when the source K and V
+        # are laid out the same way, one gather launch serves both
+        self.kv_out = torch.empty((n_kv_out, 2, n_kv_heads, kv_budget, head_dim), dtype=dtype, device=dev)
+        self.k_out = self.kv_out[:, 0]
+        self.v_out = self.kv_out[:, 1]
         self.hidden_out = (torch.empty((struct_budget, hidden_dim), dtype=torch.bfloat16, device=dev)
                            if hidden_dim else None)
         self.pos_out = torch.empty((struct_budget,), dtype=i32, device=dev)
@@ -64,8 +67,14 @@ class Prefill:
         return self.pivot
 
     # -- Algorithm 1 line 17 for one layer
-    def compact_kv(self, layer: int, k: torch.Tensor, v: torch.Tensor) -> None:
+    def compact_kv(self, layer: int, k: torch.Tensor, v: torch.Tensor,
+                   kv: Optional[torch.Tensor] = None) -> None:
+        """``kv`` (optional) is the joint storage ``[2, H_kv, N, d]`` whose halves are ``k`` and ``v``."""
         slot = layer if self.keep_kv else 0
+        if kv is not None:
+            self.ctx.compact(kv.view(2 * self.Hkv, kv.shape[2], self.d), self.i_kv[layer],
+                             self.kv_out[slot].view(2 * self.Hkv, self.kv_budget, self.d))
+            return
         self.ctx.compact(k, self.i_kv[layer], self.k_out[slot])
         self.ctx.compact(v, self.i_kv[layer], self.v_out[slot])
 
@@ -82,7 +91,7 @@ class Prefill:
         self.detect_and_select(len(layers))
         for l, t in enumerate(layers):
             if "v" in t:
-                self.compact_kv(l, t["k"], t["v"])
+                self.compact_kv(l, t["k"], t["v"], t.get("kv"))
         if hidden is not None:
             self.compact_hidden(hidden, positions)
         return self.pivot

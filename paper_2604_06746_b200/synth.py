@@ -172,11 +172,16 @@ def make_layer(wl: Workload, pl: Plan, layer: int, device: str = "cpu",
     if wl.sink:
         k[:, 0, :] *= 4.0
     st = torch_dtype(wl.dtype)
-    out = {"q_win": q.to(st).contiguous(), "k": k.to(st).contiguous(),
-           "scale": layer_scale(wl, pl, layer)}
-    del q, k
+    out = {"q_win": q.to(st).contiguous(), "scale": layer_scale(wl, pl, layer)}
     if with_v:
-        out["v"] = torch.randn((Hkv, N, d), generator=gen, device=dev, dtype=f32).to(st).contiguous()
+        # K and V of a layer share one allocation [2, H_kv, N, d] (a single gather then compacts both)
+        kv = torch.empty((2, Hkv, N, d), device=dev, dtype=st)
+        kv[0] = k.to(st)
+        del q, k
+        kv[1] = torch.randn((Hkv, N, d), generator=gen, device=dev, dtype=f32).to(st)
+        out["kv"], out["k"], out["v"] = kv, kv[0], kv[1]
+    else:
+        out["k"] = k.to(st).contiguous()
     return out
 
 
