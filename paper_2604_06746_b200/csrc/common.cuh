@@ -127,4 +127,31 @@ __device__ __forceinline__ void radix_pick_from_top(const unsigned* hist, int nb
   }
 }
 
+// Called by all threads of a 1024-thread block after a histogram pass over `nb` = 2048 bins.
+// Walks the bins from the top and finds the bin holding the `remaining`-th largest candidate;
+// writes that bin and the rank still wanted inside it.  `scratch` holds 33 words.
+__device__ __forceinline__ void block_pick_from_top(const unsigned* hist, unsigned remaining,
+                                                    unsigned* scratch, unsigned* sel_bin, unsigned* sel_rem) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b_hi = 2047 - 2 * tid, b_lo = b_hi - 1;        // this thread's two bins, higher first
+  const unsigned c_hi = hist[b_hi], c_lo = hist[b_lo];
+  const unsigned mine = c_hi + c_lo;
+  unsigned incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  __syncthreads();
+  if (lane == 31) scratch[warp] = incl;
+  __syncthreads();
+  unsigned before = incl - mine;
+  for (int w = 0; w < warp; ++w) before += scratch[w];
+  if (before < remaining && remaining <= before + mine) {
+    if (before + c_hi >= remaining) { *sel_bin = (unsigned)b_hi; *sel_rem = remaining - before; }
+    else { *sel_bin = (unsigned)b_lo; *sel_rem = remaining - before - c_hi; }
+  }
+  __syncthreads();
+}
+
 }  // namespace skv

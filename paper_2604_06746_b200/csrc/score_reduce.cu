@@ -97,14 +97,15 @@ constexpr int kHsBins = 2048;
 constexpr int kHsCopies = 8;      // each bin is kept 8 times (lane & 7) so that a warp's hits on one bin spread
 constexpr int kHsItems = 16;      // entries per thread kept in registers between the sweeps
 
-// Shared memory of head_stats: hist[kHsBins][kHsCopies] | merged[kHsBins] (dynamic, 72 KB).
+// Shared memory of head_stats: hist[kHsBins][kHsCopies] | merged[2][kHsBins] (dynamic, 80 KB).
 __global__ void __cluster_dims__(kHsCluster, 1, 1) __launch_bounds__(kHsThreads)
 head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rho,
            float* __restrict__ head_part) {
   extern __shared__ unsigned hs_smem[];
   unsigned* hist = hs_smem;                          // this CTA's counts, kHsCopies per bin
-  unsigned* merged = hs_smem + kHsBins * kHsCopies;  // cluster-wide counts (CTA 0's copy is the one used)
+  unsigned* merged = hs_smem + kHsBins * kHsCopies;  // cluster-wide counts of the two levels (CTA 0's copy counts)
   __shared__ float red[33];
+  __shared__ unsigned scan_tmp[33];
   __shared__ float slots[2 * kHsCluster];            // CTA 0: per-CTA {sum of squares, mass above}
   __shared__ unsigned sel_bin, sel_rem;
   cg::cluster_group cluster = cg::this_cluster();
@@ -117,27 +118,27 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   const bool in_regs = per <= kHsItems * kHsThreads;  // otherwise the second sweep reads memory again
   unsigned* merged0 = cluster.map_shared_rank(merged, 0);
 
-  auto clear = [&]() {
+  auto clear_local = [&]() {
     for (int b = tid; b < kHsBins * kHsCopies; b += kHsThreads) hist[b] = 0;
-    for (int b = tid; b < kHsBins; b += kHsThreads) merged[b] = 0;
   };
-  auto push = [&]() {                                // this CTA's counts into CTA 0's merged[]
+  auto push = [&](int level) {                       // this CTA's counts into CTA 0's merged[level]
     for (int b = tid; b < kHsBins; b += kHsThreads) {
       unsigned c = 0;
 #pragma unroll
       for (int k = 0; k < kHsCopies; ++k) c += hist[b * kHsCopies + k];
-      if (c) atomicAdd(&merged0[b], c);
+      if (c) atomicAdd(&merged0[level * kHsBins + b], c);
     }
   };
 
-  clear();
+  clear_local();
+  for (int b = tid; b < 2 * kHsBins; b += kHsThreads) merged[b] = 0;
   float reg[kHsItems];
 #pragma unroll
   for (int e = 0; e < kHsItems; ++e) {
     const int j = lo + e * kHsThreads + tid;
     reg[e] = (in_regs && j < hi) ? a[j] : -1.f;      // -1 marks "no entry" (real entries are >= 0)
   }
-  cluster.sync();
+  cluster.sync();                                    // every merged[] is zero before anyone pushes
   float sq = 0.f;
   if (in_regs) {
 #pragma unroll
@@ -154,18 +155,15 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
     }
   }
   __syncthreads();
-  push();
+  push(0);
   cluster.sync();
-  // copy the cluster-wide counts into this CTA (all threads, remote reads in parallel), then pick
+  // level-1 counts of the whole head: copy them here (remote reads in parallel), pick the bin
   if (rank != 0)
     for (int b = tid; b < kHsBins; b += kHsThreads) merged[b] = merged0[b];
+  clear_local();
   __syncthreads();
-  if (tid < 32) radix_pick_from_top(merged, kHsBins, (unsigned)k_rho, &sel_bin, &sel_rem);
-  __syncthreads();
+  block_pick_from_top(merged, (unsigned)k_rho, scan_tmp, &sel_bin, &sel_rem);
   const unsigned b1 = sel_bin, rem1 = sel_rem;
-  cluster.sync();                            // every CTA has read the level-1 counts
-  clear();
-  cluster.sync();
   float mass = 0.f;
   auto second = [&](float v) {
     const unsigned u = __float_as_uint(v), top = (u >> 20) & 0x7ffu;
@@ -180,7 +178,7 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
     for (int j = lo + tid; j < hi; j += kHsThreads) second(a[j]);
   }
   __syncthreads();
-  push();
+  push(1);
   const float tot_sq = block_sum_1024(sq, red);
   const float tot_mass = block_sum_1024(mass, red);
   if (tid == 0) {
@@ -190,14 +188,14 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   }
   cluster.sync();
   if (rank == 0) {
-    if (tid < 32) radix_pick_from_top(merged, kHsBins, rem1, &sel_bin, &sel_rem);
-    __syncthreads();
+    const unsigned* m2 = merged + kHsBins;
+    block_pick_from_top(m2, rem1, scan_tmp, &sel_bin, &sel_rem);
     const unsigned b2 = sel_bin, rem2 = sel_rem;
     // entries of the threshold bin above sub-bin b2, and rem2 entries of sub-bin b2 itself
     float in_bin = 0.f;
     for (int b = tid; b < kHsBins; b += kHsThreads) {
       const float mid = __uint_as_float((b1 << 20) | ((unsigned)b << 9) | 0x100u);
-      const unsigned cnt = (unsigned)b > b2 ? merged[b] : ((unsigned)b == b2 ? rem2 : 0u);
+      const unsigned cnt = (unsigned)b > b2 ? m2[b] : ((unsigned)b == b2 ? rem2 : 0u);
       in_bin = fmaf((float)cnt, mid, in_bin);
     }
     const float tot_in_bin = block_sum_1024(in_bin, red);
@@ -272,7 +270,7 @@ cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stri
   if (with_head_stats) {
     int k_rho = n / 10;
     if (k_rho < 1) k_rho = 1;
-    const int smem = (kHsBins * kHsCopies + kHsBins) * (int)sizeof(unsigned);
+    const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
     cudaError_t e = cudaFuncSetAttribute(head_stats, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     head_stats<<<ctx.cfg.n_q_heads * kHsCluster, kHsThreads, smem, st>>>(cols, col_stride, n, k_rho,

@@ -28,14 +28,14 @@ __device__ __forceinline__ unsigned order_key(float v) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Shared memory (dynamic): hist[kSelBins][kSelCopies] | merged[kSelBins].
+// Shared memory (dynamic): hist[kSelBins][kSelCopies] | merged[3][kSelBins] (one per level).
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 select_topk(const float* __restrict__ scores, long long row_stride, int n, int budget, int window,
             int* __restrict__ idx_out) {
   extern __shared__ unsigned sel_smem[];
   unsigned* hist = sel_smem;
   unsigned* merged = sel_smem + kSelBins * kSelCopies;
-  __shared__ unsigned warp_tot[32];
+  __shared__ unsigned warp_tot[33];
   __shared__ unsigned cta_gt[kSelCluster], cta_eq[kSelCluster];
   __shared__ unsigned sel_bin, sel_rem;
   cg::cluster_group cluster = cg::this_cluster();
@@ -62,10 +62,11 @@ select_topk(const float* __restrict__ scores, long long row_stride, int n, int b
     unsigned prefix = 0, prefix_mask = 0, remaining = (unsigned)k;
     const int shifts[3] = {21, 10, 0};
     const int widths[3] = {11, 11, 10};
+    for (int b = tid; b < 3 * kSelBins; b += kSelThreads) merged[b] = 0;
+    cluster.sync();                                  // every merged[] is zero before anyone pushes
     for (int pass = 0; pass < 3; ++pass) {
       for (int b = tid; b < kSelBins * kSelCopies; b += kSelThreads) hist[b] = 0;
-      for (int b = tid; b < kSelBins; b += kSelThreads) merged[b] = 0;
-      cluster.sync();
+      __syncthreads();
       const unsigned bmask = (1u << widths[pass]) - 1u;
       for (int j0 = lo + tid; j0 < hi; j0 += kSelThreads * kSelBatch) {
         float val[kSelBatch];
@@ -82,23 +83,22 @@ select_topk(const float* __restrict__ scores, long long row_stride, int n, int b
         }
       }
       __syncthreads();
+      unsigned* mlevel = merged + pass * kSelBins;   // bins above 2^width stay zero at the last level
       for (int b = tid; b < kSelBins; b += kSelThreads) {
         unsigned c = 0;
 #pragma unroll
         for (int q = 0; q < kSelCopies; ++q) c += hist[b * kSelCopies + q];
-        if (c) atomicAdd(&merged0[b], c);
+        if (c) atomicAdd(&merged0[pass * kSelBins + b], c);
       }
       cluster.sync();
       // copy the cluster-wide counts into this CTA (remote reads in parallel), then pick locally
       if (rank != 0)
-        for (int b = tid; b < kSelBins; b += kSelThreads) merged[b] = merged0[b];
+        for (int b = tid; b < kSelBins; b += kSelThreads) mlevel[b] = merged0[pass * kSelBins + b];
       __syncthreads();
-      if (tid < 32) radix_pick_from_top(merged, 1 << widths[pass], remaining, &sel_bin, &sel_rem);
-      __syncthreads();
+      block_pick_from_top(mlevel, remaining, warp_tot, &sel_bin, &sel_rem);
       prefix |= sel_bin << shifts[pass];
       prefix_mask |= bmask << shifts[pass];
       remaining = sel_rem;
-      cluster.sync();                                // every CTA has read the merged counts
     }
     thr = prefix;
     need_eq = remaining;
@@ -199,7 +199,7 @@ select_topk(const float* __restrict__ scores, long long row_stride, int n, int b
 
 cudaError_t launch_select(const float* scores, long long row_stride, int batch, int n, int budget,
                           int window, int* idx_out, cudaStream_t st) {
-  const int smem = (kSelBins * kSelCopies + kSelBins) * (int)sizeof(unsigned);
+  const int smem = (kSelBins * kSelCopies + 3 * kSelBins) * (int)sizeof(unsigned);
   cudaError_t e = cudaFuncSetAttribute(select_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   select_topk<<<batch * kSelCluster, kSelThreads, smem, st>>>(scores, row_stride, n, budget, window,
