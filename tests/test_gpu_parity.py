@@ -148,3 +148,72 @@ def test_results_are_deterministic(mods, cuda_device):
         outs.append((pf.s_hist.clone(), pf.metrics.clone(), pf.i_kv.clone(), pf.i_struct.clone()))
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+
+
+# ---- full-size configurations, in the launch configuration the benchmark times -------------
+# One or two layers of each full-size workload (the oracle needs seconds per layer at these
+# sizes): saliency and metrics element by element, selection under the gap rule at every
+# budget of the workload, compaction bit for bit on the selected rows.
+@pytest.mark.parametrize("name,layers", [("llama32k", (0, 17)), ("llama128k", (3,)), ("qwen64k", (5,)),
+                                         ("llama256k", (2,))])
+def test_full_size_layers(mods, cuda_device, name, layers):
+    binding, _ = mods
+    wl = synth.WORKLOADS[name]
+    pl = synth.plan(wl)
+    dt = synth.torch_dtype(wl.dtype)
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, dt, cuda_device)
+    f32 = torch.float32
+    for layer in layers:
+        t = synth.make_layer(wl, pl, layer, device=cuda_device)
+        s = torch.zeros(wl.seq, dtype=f32, device=cuda_device)
+        c = torch.full((wl.seq,), 2.0, dtype=f32, device=cuda_device)
+        m = torch.zeros(3, dtype=f32, device=cuda_device)
+        ctx.score_layer(t["q_win"], t["k"], t["scale"], s, m, c_inout=c, lam=0.5)
+        torch.cuda.synchronize()
+        assert ctx.poll_device_status() == binding.OK
+        o = O.score_layer(synth.to_f64(t["q_win"]), synth.to_f64(t["k"]), t["scale"])
+        tag = f"{name} layer {layer}"
+        P.assert_scores_close(s.cpu().numpy(), o["S"], f"{tag} S")
+        P.assert_scores_close(c.cpu().numpy(), 1.0 + o["S"], f"{tag} C = 0.5 * 2 + S")
+        for i, key in enumerate(("entropy", "sparsity", "variance")):
+            P.assert_metric_close(m[i].item(), o[key], f"{tag} {key}")
+        assert abs(s.sum().item() - wl.n_q_heads) < 1e-3 * wl.n_q_heads
+        for budget in wl.budgets:
+            idx = torch.zeros(budget, dtype=torch.int32, device=cuda_device)
+            ctx.select(s, budget, wl.window, idx)
+            torch.cuda.synchronize()
+            P.assert_selection_matches(idx.cpu().numpy(), o["S"], budget, wl.window,
+                                       O.select(o["S"], budget, wl.window), f"{tag} budget {budget}")
+            # the selection kernel alone, on the GPU's own fp32 scores: exact, ties included
+            assert np.array_equal(idx.cpu().numpy(), O.select(s.cpu().numpy(), budget, wl.window))
+        out = torch.empty((2 * wl.n_kv_heads, wl.budget, wl.head_dim), dtype=dt, device=cuda_device)
+        ctx.compact(t["kv"].view(2 * wl.n_kv_heads, wl.seq, wl.head_dim), idx, out)
+        torch.cuda.synchronize()
+        src = t["kv"].view(2 * wl.n_kv_heads, wl.seq, wl.head_dim).view(torch.int16).cpu().numpy()
+        assert np.array_equal(out.view(torch.int16).cpu().numpy(), O.compact(src, idx.cpu().numpy()))
+        del t
+    ctx.close()
+
+
+def test_hidden_state_gather_at_full_width(mods, cuda_device):
+    """Hidden states of the streamed 256K workload (width 4096, bf16) at its structural budget."""
+    binding, _ = mods
+    wl = synth.WORKLOADS["llama256k"]
+    hid, pos = synth.make_hidden(wl, device=cuda_device)
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, torch.bfloat16, cuda_device)
+    rng = np.random.default_rng(3)
+    b = wl.struct_budget()
+    idx_np = np.sort(rng.choice(wl.seq, size=b, replace=False)).astype(np.int32)
+    idx = torch.from_numpy(idx_np).to(cuda_device)
+    out = torch.empty((1, b, wl.hidden_dim), dtype=torch.bfloat16, device=cuda_device)
+    pout = torch.empty((1, b, 1), dtype=torch.int32, device=cuda_device)
+    ctx.compact(hid[None], idx, out)
+    ctx.compact(pos[None, :, None], idx, pout)
+    torch.cuda.synchronize()
+    sample = rng.choice(b, size=512, replace=False)          # rows checked bit for bit on the host
+    got = out[0][torch.from_numpy(sample).to(cuda_device)].view(torch.int16).cpu().numpy()
+    ref = hid[torch.from_numpy(idx_np[sample].astype(np.int64)).to(cuda_device)].view(torch.int16).cpu().numpy()
+    assert np.array_equal(got, ref)
+    assert torch.equal(out[0], hid[idx.long()])                # all rows, against an indexed read
+    assert np.array_equal(pout.cpu().numpy().ravel(), idx_np)
+    ctx.close()
