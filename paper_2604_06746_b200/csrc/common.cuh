@@ -86,6 +86,29 @@ cudaError_t launch_compact(const void* src, long long slab_stride, long long row
                            int row_bytes, int n_slabs, int n_rows_src, const int* idx, int n_idx,
                            void* dst, int* status, int sm_count, cudaStream_t st);
 
+// Programmatic dependent launch: a kernel launched with launch_pdl() may begin (block scheduling,
+// its own set-up) while the kernel before it in the stream is still draining.  pdl_trigger() lets
+// the next kernel begin; pdl_wait() returns once the previous kernel has completed and its
+// writes are visible, and must precede the first access to anything that kernel wrote or read.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // 2^x on the special-function unit (relative error about 2^-22; denormal results flush to 0).
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;

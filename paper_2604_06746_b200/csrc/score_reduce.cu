@@ -72,6 +72,8 @@ finalize_rows(const float4* __restrict__ row_part, int parts, int rows_pad, int 
 __global__ void reduce_columns(const float* __restrict__ cols, long long col_stride, int H, int n,
                                float lambda, float* __restrict__ s_out,
                                float* __restrict__ c_inout) {
+  pdl_trigger();
+  pdl_wait();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n) return;
   float s = 0.f;
@@ -130,8 +132,10 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
     }
   };
 
+  pdl_trigger();
   clear_local();
   for (int b = tid; b < 2 * kHsBins; b += kHsThreads) merged[b] = 0;
+  pdl_wait();                                        // the pooled columns come from the kernels before
   float reg[kHsItems];
 #pragma unroll
   for (int e = 0; e < kHsItems; ++e) {
@@ -216,6 +220,8 @@ finish_metrics(const float* __restrict__ row_ent, int rows_pad, int rows_pg_pad,
                int n_valid, const float* __restrict__ head_part, int H, int n, int with_head_stats,
                float* __restrict__ metrics) {
   __shared__ float red[33];
+  pdl_trigger();
+  pdl_wait();
   float ent = 0.f;
   for (int r = threadIdx.x; r < rows_pad; r += kFinalThreads)
     if ((r % rows_pg_pad) < rows_pg) ent += row_ent[r];
@@ -260,9 +266,8 @@ cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st) {
 
 cudaError_t launch_reduce_columns(const Ctx& ctx, const float* cols, long long col_stride, int n,
                                   float lambda, float* s_out, float* c_inout, cudaStream_t st) {
-  reduce_columns<<<(n + 255) / 256, 256, 0, st>>>(cols, col_stride, ctx.cfg.n_q_heads, n, lambda,
-                                                  s_out, c_inout);
-  return cudaGetLastError();
+  return launch_pdl(reduce_columns, dim3((n + 255) / 256), dim3(256), 0, st, cols, col_stride,
+                    ctx.cfg.n_q_heads, n, lambda, s_out, c_inout);
 }
 
 cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stride, int n,
@@ -273,17 +278,15 @@ cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stri
     const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
     cudaError_t e = cudaFuncSetAttribute(head_stats, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    head_stats<<<ctx.cfg.n_q_heads * kHsCluster, kHsThreads, smem, st>>>(cols, col_stride, n, k_rho,
-                                                                         ctx.ws.head_part);
-    e = cudaGetLastError();
+    e = launch_pdl(head_stats, dim3(ctx.cfg.n_q_heads * kHsCluster), dim3(kHsThreads), smem, st, cols,
+                   col_stride, n, k_rho, ctx.ws.head_part);
     if (e != cudaSuccess) return e;
   }
   const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
   const int rows_pg = (ctx.cfg.n_q_heads / ctx.cfg.n_kv_heads) * ctx.cfg.window;
-  finish_metrics<<<1, kFinalThreads, 0, st>>>(ctx.ws.row_ent, ctx.rows_pad, rows_pg_pad, rows_pg, ctx.rows,
-                                             ctx.ws.head_part, ctx.cfg.n_q_heads, n, with_head_stats ? 1 : 0,
-                                             metrics);
-  return cudaGetLastError();
+  return launch_pdl(finish_metrics, dim3(1), dim3(kFinalThreads), 0, st, (const float*)ctx.ws.row_ent,
+                    ctx.rows_pad, rows_pg_pad, rows_pg, ctx.rows, (const float*)ctx.ws.head_part,
+                    ctx.cfg.n_q_heads, n, with_head_stats ? 1 : 0, metrics);
 }
 
 cudaError_t launch_accumulate(const float* s_hist, long long row_stride, int pivot, int n,

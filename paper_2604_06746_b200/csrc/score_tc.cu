@@ -264,6 +264,12 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // The next kernel of the stream may start its set-up now.  Pass 1 reads tensors an earlier
+  // kernel may have produced and overwrites statistics the previous layer still reads: it waits
+  // here.  In pass 2 only the compute warps depend on pass 1 (the row statistics); the loads of K
+  // and Q and the MMAs start at once.
+  pdl_trigger();
+  if (PASS == 1) pdl_wait();
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -436,6 +442,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       //   lse2 = M + log2 Zt,   entropy = ln2 (log2 Zt - Xt / Zt)                (Eq. 4, one row)
       // lse_s holds -lse2; padded rows get -inf so that they contribute 2^(-inf) = 0.
       {
+        pdl_wait();
         const int ct = (int)threadIdx.x - 64;
         const int r = ct & (kRowBlock - 1), hp = ct >> 8;
         const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
@@ -591,8 +598,7 @@ cudaError_t launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const TcPar
   auto kern = tc_score<D, PASS, W>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::kAlloc);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kTcThreads, Smem<D>::kAlloc, st>>>(mq, mk, p);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(kTcThreads), Smem<D>::kAlloc, st, mq, mk, p);
 }
 
 template <int D, int PASS>
