@@ -310,6 +310,27 @@ def main():
         phase_ms["compact"] += e[2].elapsed_time(e[3])
     assert pf.ctx.poll_device_status() == binding.OK
     ms = max_over_ranks(ms, dev, world)
+    # rows beyond the core path (block-level aggregation for paged KV, attention-mass recovery)
+    bs = 16
+    blk = torch.zeros(((wl.seq + bs - 1) // bs,), dtype=torch.float32, device=dev)
+    rec = torch.zeros((wl.n_layers,), dtype=torch.float32, device=dev)
+    ex = [ev() for _ in range(3)]
+    pf.ctx.block_scores(pf.c_star, bs, blk)
+    pf.ctx.mass_recovery(pf.s_hist, pf.i_struct, rec)
+    torch.cuda.synchronize()
+    reps = 200                       # short kernels: enough launches queued that the host stays ahead
+    ex[0].record()
+    for it in range(reps):
+        pf.ctx.block_scores(pf.c_star, bs, blk)
+    ex[1].record()
+    for it in range(reps):
+        pf.ctx.mass_recovery(pf.s_hist, pf.i_struct, rec)
+    ex[2].record()
+    torch.cuda.synchronize()
+    next_rows = {"block_scores_us": ex[0].elapsed_time(ex[1]) * 1e3 / reps, "block_size": bs,
+                 "mass_recovery_us": ex[1].elapsed_time(ex[2]) * 1e3 / reps,
+                 "note": "back-to-back launches from Python; a floor of a few us per call is host launch cost",
+                 "mass_recovery_of_i_struct_min_over_layers": float(rec.min().item())}
     e2e = None if args.no_e2e else measure_e2e(wl, pf, layers, hidden, positions, dev, args.e2e_steps, world)
     assert pf.ctx.poll_device_status() == binding.OK
     if rank != 0:
@@ -350,7 +371,7 @@ def main():
             "data": "synthetic", "config": workload_config(wl, kv_budget), "pivot": pf.pivot,
             "phase_ms_per_step": {k: v / args.steps for k, v in phase_ms.items()},
             "roofline": roof, "compaction": compaction, "clocks": clocks,
-            "gpu_launches": n_launch * args.steps, "e2e": e2e}
+            "gpu_launches": n_launch * args.steps, "e2e": e2e, "next_rows": next_rows}
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, pl, kv_budget, n_layers_sample=1)
     print(json.dumps(line))

@@ -221,6 +221,39 @@ structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long s
                                  int n_rows_src, const int* idx, int n_idx, void* dst,
                                  void* stream);
 
+/*
+ * Block-Level Aggregation for block-based KV memory managers.  Paper: Section 4.1,
+ * implementation details: the importance of physical block k is the sum of the token scores
+ * (the Global In-Degree Centrality) inside it, S_block_k = sum_{t in block_k} C[t]; blocks with
+ * the lowest scores are evicted.  Block k covers tokens [k*block_size, min(n, (k+1)*block_size));
+ * the last block may be ragged.  Block-granular selection and gathering then go through
+ * structkv_select (scores = block scores, budget and window counted in blocks) and
+ * structkv_compact (row = one block of one KV head, when n is a multiple of block_size).
+ *
+ *   scores           device, fp32, vector b starts at scores + b*row_stride (elements).
+ *   block_scores_out device, [batch, ceil(n / block_size)] fp32.
+ * Sums run in token order in fp32.  Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_block_scores(structkv_ctx* ctx, const float* scores, long long row_stride,
+                                      int batch, int n, int block_size, float* block_scores_out,
+                                      void* stream);
+
+/*
+ * Attention-mass recovery of a retained token set.  Paper: Section 4.4, "Fidelity of Hidden
+ * States": the share of the original attention weights covered by the retained tokens, per
+ * layer.  With the window attention of Eq. 1-2 every row sums to 1, so for layer l the share is
+ * sum_{j in idx} S^(l)_j / sum_j S^(l)_j.
+ *
+ *   scores       device, fp32, one saliency vector per layer, vector b at scores + b*row_stride.
+ *   idx          device, [n_idx] int32 retained positions in [0, n); an out-of-range index adds
+ *                nothing and records STRUCTKV_ERR_INVALID_ARG in the device status word.
+ *   recovery_out device, [batch] fp32.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_mass_recovery(structkv_ctx* ctx, const float* scores, long long row_stride,
+                                       int batch, int n, const int* idx, int n_idx, float* recovery_out,
+                                       void* stream);
+
 /* Reads and clears the device status word (bounded-wait expiry, bad gather index).
  * Synchronises `stream`.  Returns STRUCTKV_OK if nothing was recorded. */
 structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream);

@@ -10,7 +10,7 @@ written out in NumPy float64 (a library matmul / sort serves as a step; nothing
 is blocked, fused or reordered).  Inputs are the stored bits of the tensors
 (fp32 / bf16) widened exactly to float64.
 
-Parity pins: every function below is pinned by the CPU test-suite against
+Parity pins: every function below (the two diagnostics / paged-KV helpers included) is pinned by the CPU test-suite against
 closed forms, invariants, library routines or brute force (none is unpinned).
 
 Readings of the paper where its text is silent, ambiguous or garbled
@@ -188,6 +188,28 @@ def select(scores: np.ndarray, budget: int, window: int) -> np.ndarray:
 def compact(src: np.ndarray, idx: np.ndarray) -> np.ndarray:
     """``dst[g, r, ...] = src[g, idx[r], ...]`` for ``src [n_slabs, n_rows, ...]``."""
     return np.ascontiguousarray(np.asarray(src)[:, np.asarray(idx, dtype=np.int64)])
+
+
+# ------------------------------------ Section 4.1 (implementation details): paged KV
+def block_scores(scores: np.ndarray, block_size: int) -> np.ndarray:
+    """Block-Level Aggregation: ``S_block_k = sum_{t in block_k} C[t]`` with block ``k`` =
+    tokens ``[k*block_size, (k+1)*block_size)`` (the last block may be ragged)."""
+    scores = np.asarray(scores, dtype=np.float64)
+    n = scores.shape[0]
+    n_blocks = -(-n // int(block_size))
+    out = np.zeros(n_blocks, dtype=np.float64)
+    for k in range(n_blocks):
+        out[k] = scores[k * block_size:(k + 1) * block_size].sum()
+    return out
+
+
+# ------------------------------------------- Section 4.4, "Fidelity of Hidden States"
+def mass_recovery(scores: np.ndarray, idx: np.ndarray) -> float:
+    """Share of the attention weights covered by the retained tokens ``idx``: every window
+    row of Eq. 1 sums to 1, so the share over all heads and window rows of a layer is
+    ``sum_{j in idx} S_j / sum_j S_j``."""
+    scores = np.asarray(scores, dtype=np.float64)
+    return float(scores[np.asarray(idx, dtype=np.int64)].sum() / scores.sum())
 
 
 # ------------------------------------------------------------------- Algorithm 1

@@ -61,6 +61,10 @@ lib.structkv_select.restype = _i
 lib.structkv_select.argtypes = [_vp, _vp, _ll, _i, _i, _i, _i, _vp, _vp]
 lib.structkv_compact.restype = _i
 lib.structkv_compact.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _i, _vp, _i, _vp, _vp]
+lib.structkv_block_scores.restype = _i
+lib.structkv_block_scores.argtypes = [_vp, _vp, _ll, _i, _i, _i, _vp, _vp]
+lib.structkv_mass_recovery.restype = _i
+lib.structkv_mass_recovery.argtypes = [_vp, _vp, _ll, _i, _i, _vp, _i, _vp, _vp]
 lib.structkv_poll_device_status.restype = _i
 lib.structkv_poll_device_status.argtypes = [_vp, _vp]
 
@@ -198,6 +202,25 @@ class Context:
         _check(lib.structkv_compact(self._h, src.data_ptr(), src.stride(0) * es, src.stride(1) * es,
                                     row_elems * es, src.shape[0], src.shape[1], idx.data_ptr(),
                                     idx.numel(), dst.data_ptr(), _stream(stream)), "structkv_compact")
+
+    def block_scores(self, scores: torch.Tensor, block_size: int, out: torch.Tensor,
+                     stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_block_scores over ``scores [batch, n]`` (or ``[n]``) into ``out [batch, ceil(n / block_size)]``."""
+        s2 = scores if scores.dim() == 2 else scores[None]
+        assert s2.stride(1) == 1 and s2.dtype == torch.float32 and out.dtype == torch.float32 and out.is_contiguous()
+        assert out.numel() == s2.shape[0] * ((s2.shape[1] + block_size - 1) // block_size)
+        _check(lib.structkv_block_scores(self._h, s2.data_ptr(), s2.stride(0), s2.shape[0], s2.shape[1], block_size,
+                                         out.data_ptr(), _stream(stream)), "structkv_block_scores")
+
+    def mass_recovery(self, scores: torch.Tensor, idx: torch.Tensor, out: torch.Tensor,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_mass_recovery: share of each row of ``scores [batch, n]`` that lies at ``idx``."""
+        s2 = scores if scores.dim() == 2 else scores[None]
+        assert s2.stride(1) == 1 and s2.dtype == torch.float32 and idx.dtype == torch.int32 and idx.is_contiguous()
+        assert out.dtype == torch.float32 and out.numel() == s2.shape[0]
+        _check(lib.structkv_mass_recovery(self._h, s2.data_ptr(), s2.stride(0), s2.shape[0], s2.shape[1],
+                                          idx.data_ptr(), idx.numel(), out.data_ptr(), _stream(stream)),
+               "structkv_mass_recovery")
 
     def poll_device_status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
         return lib.structkv_poll_device_status(self._h, _stream(stream))

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libstructkv.so")
-SOURCES = ["api.cu", "score_simt.cu", "score_tc.cu", "score_reduce.cu", "select.cu", "compact.cu"]
+SOURCES = ["api.cu", "score_simt.cu", "score_tc.cu", "score_reduce.cu", "select.cu", "compact.cu", "aggregate.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Wno-deprecated-gpu-targets"]
 

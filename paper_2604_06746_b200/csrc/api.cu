@@ -238,6 +238,26 @@ structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long s
              : STRUCTKV_ERR_CUDA;
 }
 
+structkv_status structkv_block_scores(structkv_ctx* ctx, const float* scores, long long row_stride,
+                                      int batch, int n, int block_size, float* block_scores_out,
+                                      void* stream) {
+  if (!ctx || !scores || !block_scores_out) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch < 1 || batch > 65535 || n < 1 || block_size < 1) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch > 1 && row_stride < n) return STRUCTKV_ERR_INVALID_ARG;
+  return launch_block_scores(scores, row_stride, batch, n, block_size, block_scores_out,
+                             (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_mass_recovery(structkv_ctx* ctx, const float* scores, long long row_stride,
+                                       int batch, int n, const int* idx, int n_idx, float* recovery_out,
+                                       void* stream) {
+  if (!ctx || !scores || !idx || !recovery_out) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch < 1 || n < 1 || n_idx < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch > 1 && row_stride < n) return STRUCTKV_ERR_INVALID_ARG;
+  return launch_mass_recovery(scores, row_stride, batch, n, idx, n_idx, recovery_out, ctx->c.ws.status,
+                              (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
+}
+
 structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream) {
   if (!ctx) return STRUCTKV_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;

@@ -82,6 +82,11 @@ cudaError_t launch_accumulate(const float* s_hist, long long row_stride, int piv
 cudaError_t launch_select(const float* scores, long long row_stride, int batch, int n, int budget,
                           int window, int* idx_out, cudaStream_t st);
 
+cudaError_t launch_block_scores(const float* scores, long long row_stride, int batch, int n, int block_size,
+                                float* out, cudaStream_t st);
+cudaError_t launch_mass_recovery(const float* scores, long long row_stride, int batch, int n, const int* idx,
+                                 int n_idx, float* out, int* status, cudaStream_t st);
+
 cudaError_t launch_compact(const void* src, long long slab_stride, long long row_stride,
                            int row_bytes, int n_slabs, int n_rows_src, const int* idx, int n_idx,
                            void* dst, int* status, int sm_count, cudaStream_t st);
