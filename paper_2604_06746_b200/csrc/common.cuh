@@ -121,40 +121,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// Adds one count per candidate lane to hist[bin]; lanes of a warp that hit the same bin are
-// merged into one shared-memory atomic (the values of one vector crowd into few bins).
-__device__ __forceinline__ void hist_add(unsigned* hist, unsigned bin, bool cand) {
-  const unsigned key = cand ? bin : 0xffffffffu;
-  const unsigned peers = __match_any_sync(0xffffffffu, key);
-  if (cand && (threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
-}
-
-// Called by the 32 lanes of warp 0 after a histogram pass.  Walks the `nb` bins (a multiple of
-// 32) from the top and finds the bin holding the `remaining`-th largest candidate; writes that
-// bin and the rank still wanted inside it.
-__device__ __forceinline__ void radix_pick_from_top(const unsigned* hist, int nb, unsigned remaining,
-                                                    unsigned* sel_bin, unsigned* sel_rem) {
-  const int lane = threadIdx.x & 31, per = nb / 32;
-  unsigned mine = 0;
-  for (int b = 0; b < per; ++b) mine += hist[nb - 1 - (lane * per + b)];
-  unsigned incl = mine;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  const unsigned before = incl - mine;
-  if (before < remaining && remaining <= incl) {
-    unsigned run = before;
-    for (int b = 0; b < per; ++b) {
-      const int bin = nb - 1 - (lane * per + b);
-      const unsigned c = hist[bin];
-      if (run + c >= remaining) { *sel_bin = (unsigned)bin; *sel_rem = remaining - run; break; }
-      run += c;
-    }
-  }
-}
-
 // Called by all threads of a 1024-thread block after a histogram pass over `nb` = 2048 bins.
 // Walks the bins from the top and finds the bin holding the `remaining`-th largest candidate;
 // writes that bin and the rank still wanted inside it.  `scratch` holds 33 words.
