@@ -143,8 +143,18 @@ def measure_e2e(wl, pf, layers, hidden, positions, dev, steps, world):
     and copies the results (compacted K / V, gathered hidden states and positions, both index sets,
     the metric table) back to pinned host memory.  One stream, copies inside the timed region."""
     host_layers = []
+    # pinned host memory is shared by the ranks of the node: stay within half of it.  With fewer
+    # host buffers than layers, layer l is copied from buffer l mod k (same bytes, same copies).
+    layer_bytes = sum(layers[0][k].numel() * layers[0][k].element_size() for k in ("q_win", "kv"))
     try:
-        for t in layers:
+        import psutil
+        host_total = psutil.virtual_memory().total
+    except Exception:
+        host_total = 64 << 30
+    local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
+    k_host = max(1, min(len(layers), int(0.5 * host_total / max(1, local_world) / layer_bytes)))
+    try:
+        for t in layers[:k_host]:
             host_layers.append({k: torch.empty(t[k].shape, dtype=t[k].dtype, pin_memory=True).copy_(t[k])
                                 for k in ("q_win", "kv")})
         host_hidden = torch.empty(hidden.shape, dtype=hidden.dtype, pin_memory=True).copy_(hidden)
@@ -154,12 +164,13 @@ def measure_e2e(wl, pf, layers, hidden, positions, dev, steps, world):
         host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
     except RuntimeError as e:
         return {"value": None, "unit": UNIT, "unavailable": f"pinned host allocation failed: {e}"[:200]}
-    h2d = sum(sum(t[k].numel() * t[k].element_size() for k in t) for t in host_layers) \
+    h2d = layer_bytes * len(layers) \
         + host_hidden.numel() * host_hidden.element_size() + host_pos.numel() * host_pos.element_size()
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
 
     def step():
-        for l, (hd, t) in enumerate(zip(host_layers, layers)):
+        for l, t in enumerate(layers):
+            hd = host_layers[l % k_host]
             for k in ("q_win", "kv"):
                 t[k].copy_(hd[k], non_blocking=True)
             pf.score(l, t["q_win"], t["k"], t["scale"])
@@ -184,7 +195,9 @@ def measure_e2e(wl, pf, layers, hidden, positions, dev, steps, world):
     ms = max_over_ranks(ms, dev, world)
     return {"value": job_tokens_per_second(wl.seq, world, ms), "unit": UNIT, "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-            "note": "inputs in pinned host memory, copied every step; results copied back to pinned host memory"}
+            "note": "inputs in pinned host memory, copied every step; results copied back to pinned host memory"
+                    + ("" if k_host == len(layers) else f"; host buffers for {k_host} of {len(layers)} layers "
+                       "(layer l is copied from buffer l mod k: half of the host memory is shared by the ranks)")}
 
 
 def run_reference(args):
