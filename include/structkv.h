@@ -222,6 +222,31 @@ structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long s
                                  void* stream);
 
 /*
+ * Per-KV-group saliency and per-slab gathers: the per-head variant of the cache selection.
+ * Paper: Section 3.2, the sentence before Eq. 2 (attention is aggregated over the query heads
+ * that share a KV head); Eq. 13 applied per KV head instead of per layer; and Section 4.1, the
+ * masked state transition for batches whose sequences carry different index sets.
+ *
+ * structkv_group_saliency: group_out[g, j] = sum over the G = H / H_kv query heads h of KV group
+ * g of head_cols[h, j], where head_cols is the pooled per-head attention written by
+ * structkv_score_layer (head_cols_out).  Summing group_out over g gives S^(l).
+ *   head_cols device, [H, n] fp32 rows col_stride apart (elements);  group_out device, [H_kv, n].
+ *
+ * structkv_compact_per_slab: structkv_compact with one index list per slab,
+ * dst[s, r, :] = src[s, idx[s*idx_slab_stride + r], :]  (idx_slab_stride >= n_idx, in elements):
+ * one list per KV head (lists from structkv_select over group_out), or one list per sequence
+ * of a batch.  All other arguments, the out-of-range rule and the byte exactness are those of
+ * structkv_compact.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_group_saliency(structkv_ctx* ctx, const float* head_cols, long long col_stride,
+                                        int n, float* group_out, void* stream);
+structkv_status structkv_compact_per_slab(structkv_ctx* ctx, const void* src, long long slab_stride_bytes,
+                                          long long row_stride_bytes, int row_bytes, int n_slabs,
+                                          int n_rows_src, const int* idx, long long idx_slab_stride,
+                                          int n_idx, void* dst, void* stream);
+
+/*
  * Block-Level Aggregation for block-based KV memory managers.  Paper: Section 4.1,
  * implementation details: the importance of physical block k is the sum of the token scores
  * (the Global In-Degree Centrality) inside it, S_block_k = sum_{t in block_k} C[t]; blocks with

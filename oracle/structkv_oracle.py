@@ -190,6 +190,26 @@ def compact(src: np.ndarray, idx: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(src)[:, np.asarray(idx, dtype=np.int64)])
 
 
+# ------------------------------------------ Section 3.2: aggregation inside a GQA group
+def group_saliency(head_cols: np.ndarray, group: int) -> np.ndarray:
+    """Pooled attention summed over the ``group`` query heads that share a KV head:
+    ``out[g, j] = sum_{h in group g} abar^{(h)}_j``; summing over ``g`` gives Eq. 2."""
+    head_cols = np.asarray(head_cols, dtype=np.float64)
+    H, n = head_cols.shape
+    assert H % group == 0
+    out = np.zeros((H // group, n), dtype=np.float64)
+    for h in range(H):
+        out[h // group] += head_cols[h]
+    return out
+
+
+def compact_per_slab(src: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """``dst[s, r, ...] = src[s, idx[s, r], ...]``: one index list per slab (per KV head, or per
+    sequence of a batch)."""
+    src, idx = np.asarray(src), np.asarray(idx, dtype=np.int64)
+    return np.stack([src[s][idx[s]] for s in range(src.shape[0])])
+
+
 # ------------------------------------ Section 4.1 (implementation details): paged KV
 def block_scores(scores: np.ndarray, block_size: int) -> np.ndarray:
     """Block-Level Aggregation: ``S_block_k = sum_{t in block_k} C[t]`` with block ``k`` =

@@ -61,6 +61,10 @@ lib.structkv_select.restype = _i
 lib.structkv_select.argtypes = [_vp, _vp, _ll, _i, _i, _i, _i, _vp, _vp]
 lib.structkv_compact.restype = _i
 lib.structkv_compact.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _i, _vp, _i, _vp, _vp]
+lib.structkv_group_saliency.restype = _i
+lib.structkv_group_saliency.argtypes = [_vp, _vp, _ll, _i, _vp, _vp]
+lib.structkv_compact_per_slab.restype = _i
+lib.structkv_compact_per_slab.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _i, _vp, _ll, _i, _vp, _vp]
 lib.structkv_block_scores.restype = _i
 lib.structkv_block_scores.argtypes = [_vp, _vp, _ll, _i, _i, _i, _vp, _vp]
 lib.structkv_mass_recovery.restype = _i
@@ -202,6 +206,28 @@ class Context:
         _check(lib.structkv_compact(self._h, src.data_ptr(), src.stride(0) * es, src.stride(1) * es,
                                     row_elems * es, src.shape[0], src.shape[1], idx.data_ptr(),
                                     idx.numel(), dst.data_ptr(), _stream(stream)), "structkv_compact")
+
+    def group_saliency(self, head_cols: torch.Tensor, out: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_group_saliency: ``head_cols [H, n]`` -> ``out [H_kv, n]`` (sum over each GQA group)."""
+        assert head_cols.stride(1) == 1 and head_cols.dtype == torch.float32 and out.is_contiguous()
+        assert head_cols.shape[0] == self.cfg.n_q_heads and out.shape == (self.cfg.n_kv_heads, head_cols.shape[1])
+        _check(lib.structkv_group_saliency(self._h, head_cols.data_ptr(), head_cols.stride(0), head_cols.shape[1],
+                                           out.data_ptr(), _stream(stream)), "structkv_group_saliency")
+
+    def compact_per_slab(self, src: torch.Tensor, idx: torch.Tensor, dst: torch.Tensor,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_compact_per_slab: ``src [n_slabs, n_rows, row...]``, ``idx [n_slabs, n_idx]`` int32."""
+        assert idx.dtype == torch.int32 and idx.dim() == 2 and idx.stride(1) == 1 and dst.is_contiguous()
+        assert idx.shape[0] == src.shape[0]
+        row_elems = 1
+        for sdim in src.shape[2:]:
+            row_elems *= sdim
+        es = src.element_size()
+        _check(lib.structkv_compact_per_slab(self._h, src.data_ptr(), src.stride(0) * es, src.stride(1) * es,
+                                             row_elems * es, src.shape[0], src.shape[1], idx.data_ptr(),
+                                             idx.stride(0), idx.shape[1], dst.data_ptr(), _stream(stream)),
+               "structkv_compact_per_slab")
 
     def block_scores(self, scores: torch.Tensor, block_size: int, out: torch.Tensor,
                      stream: Optional[torch.cuda.Stream] = None) -> None:

@@ -27,6 +27,18 @@ __global__ void block_scores(const float* __restrict__ scores, long long row_str
   out[(size_t)blockIdx.y * n_blocks + k] = acc;
 }
 
+// out[g][j] = sum of the pooled attention of the `group` query heads that share KV head g, heads
+// in ascending order.
+__global__ void group_saliency(const float* __restrict__ head_cols, long long col_stride, int group, int n,
+                               float* __restrict__ out) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  const int g = blockIdx.y;
+  float acc = 0.f;
+  for (int q = 0; q < group; ++q) acc += head_cols[(size_t)(g * group + q) * col_stride + j];
+  out[(size_t)g * n + j] = acc;
+}
+
 constexpr int kMrThreads = 1024;
 
 __device__ __forceinline__ float block_sum(float v, float* red) {
@@ -73,6 +85,12 @@ cudaError_t launch_block_scores(const float* scores, long long row_stride, int b
   const int vec4 = (block_size % 4 == 0) && ((uintptr_t)scores % 16 == 0) && (batch == 1 || row_stride % 4 == 0);
   block_scores<<<dim3((n_blocks + 127) / 128, batch), 128, 0, st>>>(scores, row_stride, n, block_size, n_blocks,
                                                                     vec4, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_group_saliency(const float* head_cols, long long col_stride, int n_heads, int group, int n,
+                                  float* out, cudaStream_t st) {
+  group_saliency<<<dim3((n + 255) / 256, n_heads / group), 256, 0, st>>>(head_cols, col_stride, group, n, out);
   return cudaGetLastError();
 }
 

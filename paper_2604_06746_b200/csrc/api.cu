@@ -232,10 +232,32 @@ structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long s
   if (row_bytes < 1 || n_slabs < 0 || n_rows_src < 1 || n_idx < 0) return STRUCTKV_ERR_INVALID_ARG;
   if (row_stride_bytes < row_bytes || slab_stride_bytes < 0) return STRUCTKV_ERR_INVALID_ARG;
   const Ctx& c = ctx->c;
-  return launch_compact(src, slab_stride_bytes, row_stride_bytes, row_bytes, n_slabs, n_rows_src, idx,
+  return launch_compact(src, slab_stride_bytes, row_stride_bytes, row_bytes, n_slabs, n_rows_src, idx, 0,
                         n_idx, dst, c.ws.status, c.sm_count, (cudaStream_t)stream) == cudaSuccess
              ? STRUCTKV_OK
              : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_compact_per_slab(structkv_ctx* ctx, const void* src, long long slab_stride_bytes,
+                                          long long row_stride_bytes, int row_bytes, int n_slabs,
+                                          int n_rows_src, const int* idx, long long idx_slab_stride,
+                                          int n_idx, void* dst, void* stream) {
+  if (!ctx || !src || !dst || !idx) return STRUCTKV_ERR_INVALID_ARG;
+  if (row_bytes < 1 || n_slabs < 0 || n_rows_src < 1 || n_idx < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if (row_stride_bytes < row_bytes || slab_stride_bytes < 0 || idx_slab_stride < n_idx)
+    return STRUCTKV_ERR_INVALID_ARG;
+  const Ctx& c = ctx->c;
+  return launch_compact(src, slab_stride_bytes, row_stride_bytes, row_bytes, n_slabs, n_rows_src, idx,
+                        idx_slab_stride, n_idx, dst, c.ws.status, c.sm_count,
+                        (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_group_saliency(structkv_ctx* ctx, const float* head_cols, long long col_stride,
+                                        int n, float* group_out, void* stream) {
+  if (!ctx || !head_cols || !group_out || n < 1 || col_stride < n) return STRUCTKV_ERR_INVALID_ARG;
+  const structkv_config& cfg = ctx->c.cfg;
+  return launch_group_saliency(head_cols, col_stride, cfg.n_q_heads, cfg.n_q_heads / cfg.n_kv_heads, n,
+                               group_out, (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
 }
 
 structkv_status structkv_block_scores(structkv_ctx* ctx, const float* scores, long long row_stride,

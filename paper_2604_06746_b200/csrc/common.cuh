@@ -88,8 +88,11 @@ cudaError_t launch_mass_recovery(const float* scores, long long row_stride, int 
                                  int n_idx, float* out, int* status, cudaStream_t st);
 
 cudaError_t launch_compact(const void* src, long long slab_stride, long long row_stride,
-                           int row_bytes, int n_slabs, int n_rows_src, const int* idx, int n_idx,
-                           void* dst, int* status, int sm_count, cudaStream_t st);
+                           int row_bytes, int n_slabs, int n_rows_src, const int* idx,
+                           long long idx_slab_stride, int n_idx, void* dst, int* status, int sm_count,
+                           cudaStream_t st);
+cudaError_t launch_group_saliency(const float* head_cols, long long col_stride, int n_heads, int group, int n,
+                                  float* out, cudaStream_t st);
 
 // Programmatic dependent launch: a kernel launched with launch_pdl() may begin (block scheduling,
 // its own set-up) while the kernel before it in the stream is still draining.  pdl_trigger() lets

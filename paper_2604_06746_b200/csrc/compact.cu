@@ -38,7 +38,8 @@ template <> __device__ __forceinline__ void st_stream<uint4>(uint4* p, const uin
 template <typename V>
 __global__ void __launch_bounds__(kCpThreads)
 gather_rows(const char* __restrict__ src, long long slab_stride, long long row_stride,
-            int units_per_row, int n_slabs, int n_rows_src, const int* __restrict__ idx, int n_idx,
+            int units_per_row, int n_slabs, int n_rows_src, const int* __restrict__ idx,
+            long long idx_slab_stride, int n_idx,
             char* __restrict__ dst, int* __restrict__ status) {
   const long long total = (long long)n_slabs * n_idx * units_per_row;
   const long long stride = (long long)gridDim.x * kCpThreads;
@@ -54,7 +55,7 @@ gather_rows(const char* __restrict__ src, long long slab_stride, long long row_s
         const long long row = u / units_per_row;           // s * n_idx + r
         const int c = (int)(u - row * units_per_row);
         const int s = (int)(row / n_idx), r = (int)(row - (long long)s * n_idx);
-        const int j = __ldg(idx + r);
+        const int j = __ldg(idx + s * idx_slab_stride + r);   // stride 0: one list for every slab
         if (j >= 0 && j < n_rows_src) {
           val[e] = ld_stream(reinterpret_cast<const V*>(src + s * slab_stride + j * row_stride +
                                                         (long long)c * sizeof(V)));
@@ -75,8 +76,9 @@ gather_rows(const char* __restrict__ src, long long slab_stride, long long row_s
 }  // namespace
 
 cudaError_t launch_compact(const void* src, long long slab_stride, long long row_stride,
-                           int row_bytes, int n_slabs, int n_rows_src, const int* idx, int n_idx,
-                           void* dst, int* status, int sm_count, cudaStream_t st) {
+                           int row_bytes, int n_slabs, int n_rows_src, const int* idx,
+                           long long idx_slab_stride, int n_idx, void* dst, int* status, int sm_count,
+                           cudaStream_t st) {
   if (n_idx == 0 || n_slabs == 0) return cudaSuccess;
   const bool a16 = ((uintptr_t)src % 16 == 0) && ((uintptr_t)dst % 16 == 0) && slab_stride % 16 == 0 &&
                    row_stride % 16 == 0 && row_bytes % 16 == 0;
@@ -93,13 +95,13 @@ cudaError_t launch_compact(const void* src, long long slab_stride, long long row
   char* d = (char*)dst;
   if (unit == 16)
     gather_rows<uint4><<<(int)blocks, kCpThreads, 0, st>>>(s, slab_stride, row_stride, upr, n_slabs,
-                                                          n_rows_src, idx, n_idx, d, status);
+                                                          n_rows_src, idx, idx_slab_stride, n_idx, d, status);
   else if (unit == 4)
     gather_rows<unsigned><<<(int)blocks, kCpThreads, 0, st>>>(s, slab_stride, row_stride, upr, n_slabs,
-                                                             n_rows_src, idx, n_idx, d, status);
+                                                             n_rows_src, idx, idx_slab_stride, n_idx, d, status);
   else
     gather_rows<unsigned char><<<(int)blocks, kCpThreads, 0, st>>>(s, slab_stride, row_stride, upr,
-                                                                  n_slabs, n_rows_src, idx, n_idx, d, status);
+                                                                  n_slabs, n_rows_src, idx, idx_slab_stride, n_idx, d, status);
   return cudaGetLastError();
 }
 

@@ -101,3 +101,52 @@ def test_centrality_recovers_more_attention_mass_than_a_single_layer_snapshot(cu
     for l in range(wl.n_layers):
         assert rec_c[l].item() == pytest.approx(O.mass_recovery(s_hist[l], pf.i_struct.cpu().numpy()), rel=1e-5)
     assert rec_c[1].item() > rec_s[1].item() and rec_c[2].item() > rec_s[2].item()
+
+
+def test_per_kv_head_selection_and_gather(cuda_device):
+    """The per-KV-head variant of the cache selection: saliency per GQA group from the pooled
+    per-head attention, one budgeted selection per KV head, one gather with a list per head."""
+    from paper_2604_06746_b200 import binding, synth
+    wl = synth.WORKLOADS["llama32k"].scaled(6000 + 13, n_layers=1, n_hubs=8, budgets=(500,))
+    pl = synth.plan(wl)
+    t = synth.make_layer(wl, pl, 0, device="cpu")
+    q, k, v = t["q_win"].to(cuda_device), t["k"].to(cuda_device), t["v"].to(cuda_device)
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, torch.bfloat16, cuda_device)
+    f32 = torch.float32
+    s = torch.zeros(wl.seq, dtype=f32, device=cuda_device)
+    m = torch.zeros(3, dtype=f32, device=cuda_device)
+    cols = torch.zeros((wl.n_q_heads, wl.seq), dtype=f32, device=cuda_device)
+    ctx.score_layer(q, k, t["scale"], s, m, head_cols_out=cols)
+    grp = torch.zeros((wl.n_kv_heads, wl.seq), dtype=f32, device=cuda_device)
+    ctx.group_saliency(cols, grp)
+    idx = torch.zeros((wl.n_kv_heads, wl.budget), dtype=torch.int32, device=cuda_device)
+    ctx.select(grp, wl.budget, wl.window, idx)
+    out_k = torch.zeros((wl.n_kv_heads, wl.budget, wl.head_dim), dtype=torch.bfloat16, device=cuda_device)
+    ctx.compact_per_slab(k, idx, out_k)
+    torch.cuda.synchronize()
+    o = O.score_layer(synth.to_f64(t["q_win"]), synth.to_f64(t["k"]), t["scale"])
+    og = O.group_saliency(o["head_cols"], wl.group)
+    P.assert_scores_close(grp.cpu().numpy(), og, "group saliency")
+    got = idx.cpu().numpy()
+    for g in range(wl.n_kv_heads):
+        P.assert_selection_matches(got[g], og[g], wl.budget, wl.window, O.select(og[g], wl.budget, wl.window),
+                                   f"KV head {g}")
+    assert len({tuple(r) for r in got.tolist()}) > 1                       # the heads do choose different tokens
+    ref = O.compact_per_slab(t["k"].view(torch.int16).numpy(), got)
+    assert np.array_equal(out_k.view(torch.int16).cpu().numpy(), ref)
+    assert ctx.poll_device_status() == binding.OK
+    ctx.close()
+
+
+def test_per_sequence_gather_of_a_batch(ctx):
+    """Masked state transition of a batch: every sequence brings its own index list (padded to a
+    common length); one launch gathers all of them, bit for bit."""
+    rng = np.random.default_rng(31)
+    B, n, width, kmax = 5, 3000, 96, 400
+    src = torch.from_numpy(rng.integers(0, 256, size=(B, n, width), dtype=np.uint8)).cuda()
+    idx_np = np.stack([np.sort(rng.choice(n, size=kmax, replace=False)) for _ in range(B)]).astype(np.int32)
+    pad = torch.from_numpy(np.concatenate([idx_np, np.zeros((B, 8), np.int32)], axis=1)).cuda()   # row stride 408
+    dst = torch.zeros((B, kmax, width), dtype=torch.uint8, device="cuda")
+    ctx.compact_per_slab(src, pad[:, :kmax], dst)
+    torch.cuda.synchronize()
+    assert np.array_equal(dst.cpu().numpy(), O.compact_per_slab(src.cpu().numpy(), idx_np))

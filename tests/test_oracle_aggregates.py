@@ -55,3 +55,30 @@ def test_mass_recovery_equals_the_row_wise_definition():
     idx = np.array([0, 5, 6, 20, 29])
     rows = [a[:, idx].sum(axis=1) for a in O.window_attention(q, k, 0.5)]
     assert O.mass_recovery(O.score_layer(q, k, 0.5)["S"], idx) == pytest.approx(np.mean(rows), rel=1e-12)
+
+
+def test_group_saliency_sums_to_eq2_and_matches_brute_force():
+    rng = np.random.default_rng(21)
+    q, k = rng.standard_normal((6, 4, 8)), rng.standard_normal((3, 25, 8))      # G = 2
+    out = O.score_layer(q, k, 0.4)
+    g = O.group_saliency(out["head_cols"], 2)
+    assert g.shape == (3, 25)
+    np.testing.assert_allclose(g.sum(axis=0), out["S"], rtol=1e-13)              # Eq. 2 is the sum over groups
+    np.testing.assert_allclose(g.sum(axis=1), 2.0, rtol=1e-12)                   # each head's pooled row sums to 1
+    for grp in range(3):                                                          # brute force over the two heads
+        np.testing.assert_allclose(g[grp], out["head_cols"][2 * grp] + out["head_cols"][2 * grp + 1], rtol=1e-15)
+    assert np.array_equal(O.group_saliency(out["head_cols"], 1), out["head_cols"])   # G = 1: identity
+    # a head only reads its own KV group: changing the keys of group 2 leaves groups 0 and 1 alone
+    k2 = k.copy(); k2[2] = rng.standard_normal((25, 8))
+    g2 = O.group_saliency(O.score_layer(q, k2, 0.4)["head_cols"], 2)
+    assert np.array_equal(g2[:2], g[:2]) and not np.allclose(g2[2], g[2])
+
+
+def test_compact_per_slab_is_a_library_take_along_axis():
+    rng = np.random.default_rng(22)
+    src = rng.integers(0, 1000, size=(3, 20, 5))
+    idx = np.stack([rng.choice(20, size=7, replace=False) for _ in range(3)])
+    got = O.compact_per_slab(src, idx)
+    assert np.array_equal(got, np.take_along_axis(src, idx[:, :, None], axis=1))
+    same = np.tile(idx[:1], (3, 1))                                               # equal lists: the shared-list gather
+    assert np.array_equal(O.compact_per_slab(src, same), O.compact(src, idx[0]))
