@@ -279,6 +279,18 @@ structkv_status structkv_mass_recovery(structkv_ctx* ctx, const float* scores, l
                                        int batch, int n, const int* idx, int n_idx, float* recovery_out,
                                        void* stream);
 
+/*
+ * Self-test of the error path every device-side wait shares (the paper has no counterpart; the
+ * conventions at the top of this header define it): launches one thread that waits, with the
+ * scorer's bounded-wait helper and a bound of `limit_cycles` SM clock cycles (1 .. 4e9), on a
+ * barrier nothing arrives on.  No copy or tensor-core work is in flight; when the bound runs out
+ * the kernel records STRUCTKV_ERR_TIMEOUT in the device status word and returns, so the next
+ * structkv_poll_device_status() reports TIMEOUT once and OK afterwards.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_selftest_wait_expiry(structkv_ctx* ctx, unsigned long long limit_cycles,
+                                              void* stream);
+
 /* Reads and clears the device status word (bounded-wait expiry, bad gather index).
  * Synchronises `stream`.  Returns STRUCTKV_OK if nothing was recorded. */
 structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream);

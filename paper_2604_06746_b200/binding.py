@@ -69,6 +69,8 @@ lib.structkv_block_scores.restype = _i
 lib.structkv_block_scores.argtypes = [_vp, _vp, _ll, _i, _i, _i, _vp, _vp]
 lib.structkv_mass_recovery.restype = _i
 lib.structkv_mass_recovery.argtypes = [_vp, _vp, _ll, _i, _i, _vp, _i, _vp, _vp]
+lib.structkv_selftest_wait_expiry.restype = _i
+lib.structkv_selftest_wait_expiry.argtypes = [_vp, ctypes.c_ulonglong, _vp]
 lib.structkv_poll_device_status.restype = _i
 lib.structkv_poll_device_status.argtypes = [_vp, _vp]
 
@@ -247,6 +249,11 @@ class Context:
         _check(lib.structkv_mass_recovery(self._h, s2.data_ptr(), s2.stride(0), s2.shape[0], s2.shape[1],
                                           idx.data_ptr(), idx.numel(), out.data_ptr(), _stream(stream)),
                "structkv_mass_recovery")
+
+    def selftest_wait_expiry(self, limit_cycles: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_selftest_wait_expiry: lets one bounded device wait run out (records TIMEOUT)."""
+        _check(lib.structkv_selftest_wait_expiry(self._h, limit_cycles, _stream(stream)),
+               "structkv_selftest_wait_expiry")
 
     def poll_device_status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
         return lib.structkv_poll_device_status(self._h, _stream(stream))

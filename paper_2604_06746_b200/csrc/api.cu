@@ -280,6 +280,14 @@ structkv_status structkv_mass_recovery(structkv_ctx* ctx, const float* scores, l
                               (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
 }
 
+structkv_status structkv_selftest_wait_expiry(structkv_ctx* ctx, unsigned long long limit_cycles,
+                                              void* stream) {
+  if (!ctx || limit_cycles == 0 || limit_cycles > 4000000000ull) return STRUCTKV_ERR_INVALID_ARG;
+  return launch_wait_probe(limit_cycles, ctx->c.ws.status, (cudaStream_t)stream) == cudaSuccess
+             ? STRUCTKV_OK
+             : STRUCTKV_ERR_CUDA;
+}
+
 structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream) {
   if (!ctx) return STRUCTKV_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;

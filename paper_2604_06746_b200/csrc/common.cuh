@@ -22,7 +22,7 @@ struct Workspace {
   float* row_lse2;      // [rows_pad] log2-domain log-sum-exp of each score row
   float* row_ent;       // [rows_pad] entropy of each score row (nats)
   float* cols;          // [H][n_pad] pooled per-head attention when the caller passes none
-  float* head_part;     // [H][4] per-head {sum of squares, top-k mass}
+  float* head_part;     // [H][4] per-head {sum of squared deviations from 1/n, top-k mass}
   size_t bytes;
 };
 
@@ -62,6 +62,10 @@ bool tc_supported(const Ctx& ctx, const ScoreArgs& a);
 structkv_status tc_create(Ctx& ctx);
 void tc_destroy(Ctx& ctx);
 cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pass, cudaStream_t st);
+
+// One thread waits (bounded by limit_cycles) on a barrier nobody arrives on, then records
+// STRUCTKV_ERR_TIMEOUT in *status.
+cudaError_t launch_wait_probe(unsigned long long limit_cycles, int* status, cudaStream_t st);
 
 // Merges the per-segment softmax statistics of every row into row_lse2 / row_ent (used by the
 // CUDA-core scorer; the tensor-core scorer does this at the start of its second pass).

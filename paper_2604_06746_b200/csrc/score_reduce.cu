@@ -82,13 +82,14 @@ __global__ void reduce_columns(const float* __restrict__ cols, long long col_str
   if (c_inout) c_inout[j] = fmaf(lambda, c_inout[j], s);
 }
 
-// Per head: sum of squares (Eq. 6) and the mass of the k_rho largest entries (Eq. 5) of the
-// pooled attention vector.  A cluster of kHsCluster CTAs shares one head; each CTA owns a slice
-// of the keys.  All entries are >= 0, so the unsigned order of the fp32 bit patterns is the
+// Per head: sum of squared deviations from 1/n (Eq. 6: the pooled vector sums to 1, so 1/n is its
+// mean; summing deviations instead of squares keeps near-uniform attention from cancelling) and
+// the mass of the k_rho largest entries (Eq. 5) of the pooled attention vector.  A cluster of
+// kHsCluster CTAs shares one head; each CTA owns a slice of the keys.  All entries are >= 0, so the unsigned order of the fp32 bit patterns is the
 // order of the values.  Two counting sweeps locate the k_rho-th largest value to 22 bits
 // (histograms are merged in CTA 0 of the cluster through distributed shared memory with
 // integer atomics, so the result does not depend on arrival order):
-//   sweep 1: histogram of bits 30..20 (exponent + 3 mantissa bits); sum of squares
+//   sweep 1: histogram of bits 30..20 (exponent + 3 mantissa bits); sum of squared deviations
 //   sweep 2: exact sum of the entries above the threshold bin (fixed order) and a histogram of
 //            bits 19..9 of the entries inside it
 // The entries inside the threshold bin are then summed as count x bin midpoint: bins of the
@@ -108,7 +109,7 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   unsigned* merged = hs_smem + kHsBins * kHsCopies;  // cluster-wide counts of the two levels (CTA 0's copy counts)
   __shared__ float red[33];
   __shared__ unsigned scan_tmp[33];
-  __shared__ float slots[2 * kHsCluster];            // CTA 0: per-CTA {sum of squares, mass above}
+  __shared__ float slots[2 * kHsCluster];            // CTA 0: per-CTA {sum of squared deviations, mass above}
   __shared__ unsigned sel_bin, sel_rem;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -144,17 +145,20 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   }
   cluster.sync();                                    // every merged[] is zero before anyone pushes
   float sq = 0.f;
+  const float mean = 1.f / (float)n;
   if (in_regs) {
 #pragma unroll
     for (int e = 0; e < kHsItems; ++e)
       if (reg[e] >= 0.f) {
-        sq = fmaf(reg[e], reg[e], sq);
+        const float dv = reg[e] - mean;
+        sq = fmaf(dv, dv, sq);
         atomicAdd(&hist[((__float_as_uint(reg[e]) >> 20) & 0x7ffu) * kHsCopies + copy], 1u);
       }
   } else {
     for (int j = lo + tid; j < hi; j += kHsThreads) {
       const float v = a[j];
-      sq = fmaf(v, v, sq);
+      const float dv = v - mean;
+      sq = fmaf(dv, dv, sq);
       atomicAdd(&hist[((__float_as_uint(v) >> 20) & 0x7ffu) * kHsCopies + copy], 1u);
     }
   }
@@ -213,7 +217,7 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
 }
 
 // metrics[0] = mean entropy of the valid score rows (Eq. 4);  metrics[1] = mean_h top-mass
-// (Eq. 5);  metrics[2] = mean_h (sum_sq / n - 1 / n^2) (Eq. 6; rows sum to 1).  With head
+// (Eq. 5);  metrics[2] = mean_h (sum of squared deviations from 1/n) / n (Eq. 6).  With head
 // statistics disabled metrics[1..2] are NaN.  One block, fixed summation order.
 __global__ void __launch_bounds__(kFinalThreads)
 finish_metrics(const float* __restrict__ row_ent, int rows_pad, int rows_pg_pad, int rows_pg,
@@ -237,7 +241,7 @@ finish_metrics(const float* __restrict__ row_ent, int rows_pad, int rows_pg_pad,
   const float inv_n = 1.f / (float)n;
   for (int h = 0; h < H; ++h) {
     rho += head_part[h * 4 + 1];
-    var += head_part[h * 4 + 0] * inv_n - inv_n * inv_n;
+    var += head_part[h * 4 + 0] * inv_n;
   }
   metrics[1] = rho / (float)H;
   metrics[2] = var / (float)H;

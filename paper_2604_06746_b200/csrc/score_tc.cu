@@ -5,14 +5,19 @@
 //   pass 1  D[rows, keys] = Q K^T     lane = score row  -> per-row (ref, Z, U) over a key segment
 //   pass 2  D[keys, rows] = K Q^T     lane = key        -> per-head column sums for every key
 //
-// so both reductions are loops inside one thread (no shuffles).  A work unit is (KV group g,
-// row block rb of up to 256 score rows); the key range of a unit is split into `segs` equal
-// segments, one CTA each.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the
+// so both reductions are loops inside one thread (no shuffles).  Both passes issue M128 x N256
+// MMAs: pass 1 multiplies one 128-row half of the Q block with a PAIR of 128-key tiles (two
+// neighbouring stages of the K ring form one 256-key operand), pass 2 one 128-key tile with the
+// whole 256-row Q block.  (An N128 MMA reads as many operand bytes from shared memory per clock
+// as the SM can deliver, and slows down as soon as anything else touches shared memory.)
+// A work unit is (KV group g, row block rb of up to 256 score rows); the key range of a unit
+// is split into `segs` equal segments, one CTA each.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the
 // tensor-memory allocation), warps 2..17 = compute (four per scheduler, so that one warp's
 // tensor-memory load latency hides behind the others' arithmetic).  Pass 2 starts by merging
 // the segments' row statistics into each row's log-sum-exp (and, in segment 0, its entropy).
-// Every wait is bounded; on expiry the CTA records STRUCTKV_ERR_TIMEOUT, stops, drains its
-// own copies and frees tensor memory.
+// Every wait is bounded; on expiry the CTA records STRUCTKV_ERR_TIMEOUT and stops issuing work;
+// it then waits (with a fresh bound that ignores the abort flag) for its own copies and MMAs in
+// flight, and frees tensor memory only if those MMAs are known to have retired.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -30,9 +35,9 @@ constexpr unsigned long long kWaitCycles = 1000000000ull;   // about 0.5 s at th
 constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 0 * x stays finite
 
 struct TcParams {
-  int n_keys, window, group, rows_pg, rows_pg_pad, rows_pad, n_rb, segs, n_tiles;
+  int n_keys, window, group, rows_pg, rows_pg_pad, rows_pad, n_rb, segs, n_tiles, n_pairs;
   float c2;                            // scale * log2(e)
-  float4* row_part;                    // pass 1 out, pass 2 in: [2 * segs][rows_pad] (ref, Z, U, -)
+  float4* row_part;                    // pass 1 out, pass 2 in: [segs][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride]
   long long col_stride;
@@ -65,8 +70,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the barrier did not flip in time or the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  Returns false if the barrier did not flip within `limit` cycles or the CTA is
+// aborting; the first waiter whose bound expires raises the CTA's abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit = kWaitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -74,7 +81,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 256; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if ((unsigned long long)(clock64() - t0) > kWaitCycles) { *abort_flag = 1; return false; }
+    if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return false; }
+  }
+}
+// Bounded wait for work this thread itself put in flight (copies, MMAs): runs after an abort as
+// well, so it ignores the abort flag and starts its own timer.  False = still in flight.
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                           unsigned long long limit = kWaitCycles) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return false; }
   }
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
@@ -176,6 +196,21 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
   unpack2(x, x0, x1);
   return pack2(fast_exp2(x0), fast_exp2(x1));
 }
+// Scalar form of the same polynomial (pass 1).
+__device__ __forceinline__ float exp2_poly1(float x) {
+  x = fminf(fmaxf(x, -125.f), 126.f);
+  const float t = x + 12582912.0f;
+  const float f = x - (t - 12582912.0f);
+  float p = fmaf(0.0551716685f, f, 0.2426111251f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999280572f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// In pass 1, of every 8 consecutive elements the first kPoly1 take the polynomial.
+#ifndef SKV_POLY1
+#define SKV_POLY1 2
+#endif
+constexpr int kPoly1 = SKV_POLY1;
 // In pass 2, of every 8 consecutive element pairs the first kPoly2 take the polynomial, the
 // rest the special-function unit: the two pipes work side by side (2 of 8 measured best).
 #ifndef SKV_POLY2
@@ -204,14 +239,19 @@ template <int D>
 struct Smem {
   static constexpr int kSub = D / 64;                      // 64-column (128-byte) sub-tiles per operand
   static constexpr int kQBytes = kRowBlock * 128 * kSub;   // Q block: 256 rows
-  static constexpr int kKBytes = kKeyTile * 128 * kSub;    // one K tile: 128 keys
+  static constexpr int kKSub = kKeyTile * 128;             // one sub-tile of one K stage: 128 keys x 128 bytes
+  static constexpr int kKBytes = kKSub * kSub;             // bytes TMA delivers per stage
   static constexpr int kQOff = 0;
+  // K ring, sub-tile major: sub-tile c of stage s sits at kKOff + (c * kStages + s) * kKSub, so the
+  // same sub-tile of stages s and s + 1 is one contiguous 256-key operand
   static constexpr int kKOff = kQBytes;
   static constexpr int kLseOff = kKOff + kStages * kKBytes;          // 256 floats
-  static constexpr int kMergeOff = kLseOff + kRowBlock * 4;          // 256 x (M, Z, X) for the pass-2 merge
-  static constexpr int kBarOff = kMergeOff + kRowBlock * 16;
+  // pass 1: [4 column groups][256 rows] (ref, Z, U); pass 2: 256 x (M, Z, X) for the merge
+  static constexpr int kMergeOff = kLseOff + kRowBlock * 4;
+  static constexpr int kBarOff = kMergeOff + 4 * kRowBlock * 16;
   static constexpr int kBytes = kBarOff + 256;
   static constexpr int kAlloc = kBytes + 1024;             // slack to align the base to 1024 bytes
+  static_assert(kAlloc <= 227 * 1024, "shared memory of one CTA");
 };
 
 // Barrier slots (8 bytes each) inside the barrier area.
@@ -232,15 +272,18 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   float* lse_s = reinterpret_cast<float*>(sm + L::kLseOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kBarOff + 8 * kBarCount);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + L::kBarOff + 8 * kBarCount + 8);
+  volatile int* mma_in_flight = reinterpret_cast<volatile int*>(sm + L::kBarOff + 8 * kBarCount + 16);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int unit = blockIdx.x / p.segs, seg = blockIdx.x - unit * p.segs;
   const int g = unit / p.n_rb, rb = unit - g * p.n_rb;
-  const int t_lo = (int)((long long)seg * p.n_tiles / p.segs);
-  const int t_hi = (int)((long long)(seg + 1) * p.n_tiles / p.segs);
+  // Pass 1 walks its segment in pairs of key tiles (256 keys per MMA), pass 2 in single tiles.
+  const int n_items = PASS == 1 ? p.n_pairs : p.n_tiles;
+  const int t_lo = (int)((long long)seg * n_items / p.segs);
+  const int t_hi = (int)((long long)(seg + 1) * n_items / p.segs);
   const int n_my = t_hi - t_lo;
-  // Pass 1 sweeps its key tiles forward, pass 2 backward: the tiles pass 1 touched last are
-  // the ones still in L2 when pass 2 starts.
+  // Pass 1 sweeps forward, pass 2 backward: the tiles pass 1 touched last are the ones still
+  // in L2 when pass 2 starts.
   auto tile_of = [&](int t) { return PASS == 1 ? t_lo + t : t_hi - 1 - t; };
   const int rows_here = min(kRowBlock, p.rows_pg - rb * kRowBlock);     // valid score rows in this block
   const int n_half = (rows_here + 127) / 128;
@@ -254,6 +297,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     }
     mbar_init(bars + 8 * kBarDrain, 1);
     *abort_flag = 0;
+    *mma_in_flight = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -264,12 +308,13 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  // The next kernel of the stream may start its set-up now.  Pass 1 reads tensors an earlier
-  // kernel may have produced and overwrites statistics the previous layer still reads: it waits
-  // here.  In pass 2 only the compute warps depend on pass 1 (the row statistics); the loads of K
-  // and Q and the MMAs start at once.
-  pdl_trigger();
+  // Pass 1 reads tensors an earlier kernel may have produced and overwrites statistics the
+  // previous layer still reads: it waits for that kernel first and only then lets pass 2 begin,
+  // so pass 2 (whose producer warps read K and Q without waiting) never runs ahead of the
+  // kernel that precedes pass 1.  In pass 2 only the compute warps depend on pass 1 (the row
+  // statistics): the loads of K and Q and the MMAs start at once.
   if (PASS == 1) pdl_wait();
+  pdl_trigger();
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -279,58 +324,83 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       for (int s = 0; s < L::kSub; ++s)
         tma_load_2d(base + L::kQOff + s * (L::kQBytes / L::kSub), &map_q, bars + 8 * kBarQ, s * 64, q_row0);
       int issued = 0;
-      for (int t = 0; t < n_my; ++t) {
+      const int n_load = PASS == 1 ? 2 * n_my : n_my;      // 128-key tiles this CTA loads
+      for (int t = 0; t < n_load; ++t) {
         const int s = t % kStages;
         const uint32_t ph = (uint32_t)(t / kStages) & 1u;
         if (!mbar_wait(bars + 8 * (kBarEmpty + s), ph ^ 1u, abort_flag)) break;
         mbar_expect_tx(bars + 8 * (kBarFull + s), L::kKBytes);
+        // a pair's second tile may lie wholly beyond the last key: TMA fills it with zeros and
+        // the causal mask discards it
+        const int tile = PASS == 1 ? 2 * t_lo + t : tile_of(t);
         for (int c = 0; c < L::kSub; ++c)
-          tma_load_3d(base + L::kKOff + s * L::kKBytes + c * (L::kKBytes / L::kSub), &map_k,
-                      bars + 8 * (kBarFull + s), c * 64, tile_of(t) * kKeyTile, g);
+          tma_load_3d(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
+                      c * 64, tile * kKeyTile, g);
         ++issued;
       }
       // drain: every copy this thread issued must have landed before the CTA may exit
-      mbar_wait(bars + 8 * kBarQ, 0, abort_flag);
+      mbar_drain(bars + 8 * kBarQ, 0, abort_flag);
       for (int t = max(0, issued - kStages); t < issued; ++t)
-        mbar_wait(bars + 8 * (kBarFull + t % kStages), (uint32_t)(t / kStages) & 1u, abort_flag);
+        mbar_drain(bars + 8 * (kBarFull + t % kStages), (uint32_t)(t / kStages) & 1u, abort_flag);
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0 && n_my > 0) {
-      constexpr uint32_t idesc = (PASS == 1) ? instr_desc(128, 128) : instr_desc(128, 256);
+      constexpr uint32_t idesc = instr_desc(128, 256);
       const uint64_t q_desc0 = smem_desc(base + L::kQOff), k_desc0 = smem_desc(base + L::kKOff);
       bool ok = mbar_wait(bars + 8 * kBarQ, 0, abort_flag);
-      int t = 0;
-      for (; ok && t < n_my; ++t) {
-        const int s = t % kStages, a = t % kAccStages;
-        if (!mbar_wait(bars + 8 * (kBarFull + s), (uint32_t)(t / kStages) & 1u, abort_flag)) break;
-        if (!mbar_wait(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(t / kAccStages) & 1u) ^ 1u, abort_flag)) break;
-        tc_fence_after();
-        // descriptors differ only in the start-address field (16-byte units, no carry out of it)
-        const uint64_t kd = k_desc0 + (uint64_t)((s * L::kKBytes) >> 4);
-        if (PASS == 1) {
-          for (int hf = 0; hf < n_half; ++hf) {
+      // descriptors differ only in the start-address field (16-byte units, no carry out of it)
+      if (PASS == 1) {
+        // unit u = (pair, row half): A = one 128-row half of Q, B = the pair's 256 keys
+        for (int t = 0, u = 0; ok && t < n_my; ++t) {
+          const int s0 = (2 * t) % kStages;
+          const uint32_t ph = (uint32_t)((2 * t) / kStages) & 1u;
+          if (!mbar_wait(bars + 8 * (kBarFull + s0), ph, abort_flag)) break;
+          if (!mbar_wait(bars + 8 * (kBarFull + s0 + 1), ph, abort_flag)) break;
+          const uint64_t kd = k_desc0 + (uint64_t)((s0 * L::kKSub) >> 4);
+          for (int hf = 0; hf < n_half; ++hf, ++u) {
+            const int a = u % kAccStages;
+            if (!mbar_wait(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(u / kAccStages) & 1u) ^ 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t qo = (kk / 4) * (L::kQBytes / L::kSub) + hf * (128 * 128) + (kk % 4) * 32;
-              const uint32_t ko = (kk / 4) * (L::kKBytes / L::kSub) + (kk % 4) * 32;
-              tc_mma_bf16(tmem + a * 256 + hf * 128, q_desc0 + (qo >> 4), kd + (ko >> 4), idesc, kk > 0);
+              const uint32_t ko = (kk / 4) * (kStages * L::kKSub) + (kk % 4) * 32;
+              tc_mma_bf16(tmem + a * 256, q_desc0 + (qo >> 4), kd + (ko >> 4), idesc, kk > 0);
             }
+            *mma_in_flight = 1;
+            tc_commit(bars + 8 * (kBarAccFull + a));   // accumulator ready for the compute warps
           }
-        } else {
+          if (!ok) break;
+          tc_commit(bars + 8 * (kBarEmpty + s0));      // both K stages reusable once these MMAs have read them
+          tc_commit(bars + 8 * (kBarEmpty + s0 + 1));
+        }
+      } else {
+        for (int t = 0; ok && t < n_my; ++t) {
+          const int s = t % kStages, a = t % kAccStages;
+          if (!mbar_wait(bars + 8 * (kBarFull + s), (uint32_t)(t / kStages) & 1u, abort_flag)) break;
+          if (!mbar_wait(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(t / kAccStages) & 1u) ^ 1u, abort_flag)) break;
+          tc_fence_after();
+          const uint64_t kd = k_desc0 + (uint64_t)((s * L::kKSub) >> 4);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t ko = (kk / 4) * (L::kKBytes / L::kSub) + (kk % 4) * 32;
+            const uint32_t ko = (kk / 4) * (kStages * L::kKSub) + (kk % 4) * 32;
             const uint32_t qo = (kk / 4) * (L::kQBytes / L::kSub) + (kk % 4) * 32;
             tc_mma_bf16(tmem + a * 256, kd + (ko >> 4), q_desc0 + (qo >> 4), idesc, kk > 0);
           }
+          *mma_in_flight = 1;
+          tc_commit(bars + 8 * (kBarEmpty + s));       // K stage reusable once these MMAs have read it
+          tc_commit(bars + 8 * (kBarAccFull + a));     // accumulator ready for the compute warps
         }
-        tc_commit(bars + 8 * (kBarEmpty + s));       // K stage reusable once these MMAs have read it
-        tc_commit(bars + 8 * (kBarAccFull + a));     // accumulator ready for the compute warps
       }
       // drain: all issued MMAs must retire before tensor memory is freed
-      tc_commit(bars + 8 * kBarDrain);
-      mbar_wait(bars + 8 * kBarDrain, 0, abort_flag);
+      if (*mma_in_flight) {
+        tc_commit(bars + 8 * kBarDrain);
+        if (mbar_drain(bars + 8 * kBarDrain, 0, abort_flag)) *mma_in_flight = 0;
+      }
     }
   } else {
     // ---------------- compute warps ----------------
@@ -359,81 +429,118 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     };
 
     if (PASS == 1) {
-      // accumulator columns [0,128) hold rows 0..127 x the tile's 128 keys, [128,256) rows 128..255;
-      // this thread owns one row and 64 of the tile's keys
-      const int half = sub & 1, ch = sub >> 1;
-      const int row_in_block = half * 128 + quarter * 32 + lane;
-      const bool row_valid = row_in_block < rows_here;
-      const bool warp_active = (half * 128 + quarter * 32) < rows_here;
-      const int i_win = (rb * kRowBlock + row_in_block) % p.window;      // window row index of this score row
-      const int t_pos = p.n_keys - p.window + i_win;                     // its position: sees keys <= t_pos
-      float ref = -INFINITY, Z = 0.f, U = 0.f;
-      // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible.
-      // (Scalar arithmetic: here the packed form measured slower, the pairs are unpacked twice.)
-      auto accumulate = [&]() {
+      // A unit's accumulator holds one 128-row half of the block x the pair's 256 keys.  This
+      // thread owns row (quarter * 32 + lane) of BOTH halves (units alternate between them) and
+      // the 64 keys [sub * 64, sub * 64 + 64) of every pair.
+      struct RowStat { float ref, Z, U; };
+      RowStat st[2] = {{-INFINITY, 0.f, 0.f}, {-INFINITY, 0.f, 0.f}};
+      const int row_lo = quarter * 32 + lane;
+      const int i_win = row_lo % p.window;          // window row of this thread's rows (the window divides 128)
+      const int t_pos = p.n_keys - p.window + i_win;                     // their position: they see keys <= t_pos
+      const int first_tail_pair = (p.n_keys - p.window + 1) / (2 * kKeyTile);
+      // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible;
+      // of every 8 elements the first kPoly1 are exponentiated on the FMA pipe
+      auto accumulate = [&](RowStat& r) {
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-          const float x = fmaf(v[e], p.c2, -ref);
-          const float pr = fast_exp2(x);
-          Z += pr;
-          U = fmaf(pr, x, U);
+          const float x = fmaf(v[e], p.c2, -r.ref);
+          const float pr = ((e & 7) < kPoly1) ? exp2_poly1(x) : fast_exp2(x);
+          r.Z += pr;
+          r.U = fmaf(pr, x, r.U);
         }
       };
       // same with the causal mask, moving the reference up to the chunk maximum first
       // (v[0] is key jb); works from registers, so the accumulator is not needed again
-      auto accumulate_careful = [&](int jb) {
+      auto accumulate_careful = [&](RowStat& r, int jb) {
         float mx = -INFINITY;
 #pragma unroll
         for (int e = 0; e < 32; ++e)
           if (jb + e <= t_pos) mx = fmaxf(mx, v[e] * p.c2);
-        if (mx > ref) {
-          if (ref != -INFINITY) {
-            const float dm = ref - mx, f = fast_exp2(dm);
-            U = f * fmaf(dm, Z, U);
-            Z = f * Z;
+        if (mx > r.ref) {
+          if (r.ref != -INFINITY) {
+            const float dm = r.ref - mx, f = fast_exp2(dm);
+            r.U = f * fmaf(dm, r.Z, r.U);
+            r.Z = f * r.Z;
           }
-          ref = mx;
+          r.ref = mx;
         }
-        const float ref_use = (ref == -INFINITY) ? 0.f : ref;      // row has seen no key yet: all masked
+        const float ref_use = (r.ref == -INFINITY) ? 0.f : r.ref;  // row has seen no key yet: all masked
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const float x = (jb + e <= t_pos) ? fmaf(v[e], p.c2, -ref_use) : kMasked;
           const float pr = fast_exp2(x);
-          Z += pr;
-          U = fmaf(pr, x, U);
+          r.Z += pr;
+          r.U = fmaf(pr, x, r.U);
         }
       };
-      // `fast` is warp-uniform: the tile is unmasked and the reference already exists
-      auto chunk = [&](int jb, bool fast) {
+      // `fast` is warp-uniform: the keys are unmasked and the reference already exists
+      auto chunk = [&](RowStat& r, int jb, bool fast) {
         if (fast) {
-          const float Z0 = Z, U0 = U;
-          accumulate();
+          const float Z0 = r.Z, U0 = r.U;
+          accumulate(r);
           // a logit far above the reference overflowed (or was clamped at 2^126): redo the chunk
-          const bool ovf = !(Z < 4.0e37f) || !(fabsf(U) < 3.0e38f);
-          if (__any_sync(0xffffffffu, ovf)) { Z = Z0; U = U0; accumulate_careful(jb); }
+          const bool ovf = !(r.Z < 4.0e37f) || !(fabsf(r.U) < 3.0e38f);
+          if (__any_sync(0xffffffffu, ovf)) { r.Z = Z0; r.U = U0; accumulate_careful(r, jb); }
         } else {
-          accumulate_careful(jb);
+          accumulate_careful(r, jb);
         }
       };
-      for (int t = 0; t < n_my; ++t) {
-        if (!acc_full(t)) break;
-        const uint32_t taddr = tmem + lane_base + (uint32_t)((t % kAccStages) * 256 + half * 128 + ch * 64);
-        const int jb = (t_lo + t) * kKeyTile + ch * 64;
-        const bool plain = (t_lo + t) < first_tail_tile;
-        if (warp_active) {
-          tmem_ld32(taddr, v);
-          tmem_ld_wait(v);
-          chunk(jb, plain && t > 0);
-          tmem_ld32(taddr + 32, v);
-          tmem_ld_wait(v);
+      bool live = true;
+      for (int t = 0, u = 0; live && t < n_my; ++t) {
+        const int jb = (t_lo + t) * (2 * kKeyTile) + sub * 64;
+        const bool plain = (t_lo + t) < first_tail_pair;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          if (hf < n_half && live) {
+            if (!acc_full(u)) { live = false; continue; }
+            const bool warp_active = (hf * 128 + quarter * 32) < rows_here;
+            const uint32_t taddr = tmem + lane_base + (uint32_t)((u % kAccStages) * 256 + sub * 64);
+            if (warp_active) {
+              tmem_ld32(taddr, v);
+              tmem_ld_wait(v);
+              chunk(st[hf], jb, plain && t > 0);
+              tmem_ld32(taddr + 32, v);
+              tmem_ld_wait(v);
+            }
+            acc_release(u);
+            if (warp_active) chunk(st[hf], jb + 32, plain);
+            ++u;
+          }
         }
-        acc_release(t);
-        if (warp_active) chunk(jb + 32, plain);
       }
-      // two partial statistics per (row, segment): one per 64-key half of the tiles
-      if (row_valid)
-        p.row_part[(size_t)(seg * 2 + ch) * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
-            n_my > 0 ? make_float4(ref, Z, U, 0.f) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
+      // The four column groups of a row fold into ONE partial per (row, segment): re-reference
+      // each to the largest reference M, Z = sum_c 2^(ref_c - M) Z_c,
+      // U = sum_c 2^(ref_c - M) (U_c + (ref_c - M) Z_c).
+      float4* part_s = reinterpret_cast<float4*>(sm + L::kMergeOff);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf)
+        part_s[sub * kRowBlock + hf * 128 + row_lo] = make_float4(st[hf].ref, st[hf].Z, st[hf].U, 0.f);
+      asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+      if (sub == 0) {
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int row_in_block = hf * 128 + row_lo;
+          if (row_in_block < rows_here) {
+            float4 c[4];
+            float M = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              c[k] = part_s[k * kRowBlock + row_in_block];
+              if (c[k].y > 0.f) M = fmaxf(M, c[k].x);
+            }
+            float Z = 0.f, U = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (c[k].y > 0.f) {
+                const float dm = c[k].x - M, f = fast_exp2(dm);
+                Z = fmaf(f, c[k].y, Z);
+                U = fmaf(f, fmaf(dm, c[k].y, c[k].z), U);
+              }
+            p.row_part[(size_t)seg * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
+                make_float4(M, Z, U, 0.f);
+          }
+        }
+      }
     } else {
       // pass 2.  First the compute threads merge the partial statistics of this block's rows,
       // two threads per row (each takes every other partial, loads batched), then one of them
@@ -446,7 +553,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         const int ct = (int)threadIdx.x - 64;
         const int r = ct & (kRowBlock - 1), hp = ct >> 8;
         const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
-        const int parts = 2 * p.segs;
+        const int parts = p.segs;
         float M = -INFINITY, Zt = 0.f, Xt = 0.f;
         auto fold = [&](float ref_s, float Z_s, float X_s) {     // X_s = sum 2^(..)(.. - ref_s), relative to ref_s
           if (!(Z_s > 0.f)) return;
@@ -586,9 +693,25 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   tc_fence_before();
   __syncthreads();
   if (*abort_flag && threadIdx.x == 0) atomicCAS(p.status, 0, (int)STRUCTKV_ERR_TIMEOUT);
-  if (warp == 1) {
+  // tensor memory is freed only when no MMA of this CTA can still write to it
+  if (warp == 1 && !*mma_in_flight) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+// Self-test of the bounded wait: one thread waits, with the scorer's own helper, on a barrier
+// that nothing will ever arrive on.  No copy, MMA or tensor-memory allocation is involved, so
+// when the bound expires the kernel simply records STRUCTKV_ERR_TIMEOUT and returns.
+__global__ void wait_expiry_probe(unsigned long long limit_cycles, int* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_word;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_word = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(smem_u32(&bar), 0, &abort_word, limit_cycles))
+      atomicCAS(status, 0, (int)STRUCTKV_ERR_TIMEOUT);
   }
 }
 
@@ -641,6 +764,11 @@ bool encode_maps(const Ctx& ctx, const ScoreArgs& a, CUtensorMap* mq, CUtensorMa
 
 }  // namespace
 
+cudaError_t launch_wait_probe(unsigned long long limit_cycles, int* status, cudaStream_t st) {
+  wait_expiry_probe<<<1, 32, 0, st>>>(limit_cycles, status);
+  return cudaGetLastError();
+}
+
 bool tc_supported(const Ctx& ctx, const ScoreArgs& a) {
   if (!ctx.tc || ctx.cfg.dtype != STRUCTKV_BF16) return false;
   const int w = ctx.cfg.window;
@@ -682,10 +810,11 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.n_rb = (p.rows_pg + kRowBlock - 1) / kRowBlock;
   p.n_tiles = (a.n_keys + kKeyTile - 1) / kKeyTile;
   const int units = ctx.cfg.n_kv_heads * p.n_rb;
+  p.n_pairs = (p.n_tiles + 1) / 2;
   int segs = ctx.sm_count / units;
   if (segs < 1) segs = 1;
-  if (segs > p.n_tiles) segs = p.n_tiles;
-  if (2 * segs > kMaxParts) segs = kMaxParts / 2;   // pass 1 leaves two partial statistics per segment
+  if (segs > p.n_pairs) segs = p.n_pairs;
+  if (segs > kMaxParts) segs = kMaxParts;           // pass 1 leaves one partial statistic per segment
   p.segs = segs;
   p.c2 = a.scale * kLog2e;
   p.row_part = ctx.ws.row_part;
@@ -693,7 +822,7 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.cols = a.cols;
   p.col_stride = a.col_stride;
   p.status = ctx.ws.status;
-  *parts_out = 2 * segs;
+  *parts_out = segs;
   const int grid = units * segs;
   const int d = ctx.cfg.head_dim, w = ctx.cfg.window;
   if (d == 128) return pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);

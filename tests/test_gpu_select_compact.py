@@ -112,3 +112,21 @@ def test_compact_flags_out_of_range_index_without_faulting(ctx):
     got = dst.cpu().numpy()[0]
     assert np.array_equal(got[[0, 1, 4]], src.cpu().numpy()[0][[0, 5, 7]])
     assert np.all(got[[2, 3]] == 255)                                 # skipped rows stay untouched
+
+
+def test_bounded_wait_expiry_is_reported_once(cuda_device):
+    """A device-side wait whose bound runs out records TIMEOUT in the status word and returns:
+    the poll reports it once, the context stays usable and later polls are clean."""
+    from paper_2604_06746_b200 import binding
+    ctx = binding.Context(8, 2, 64, 32, 2048, torch.float32, cuda_device)
+    assert ctx.poll_device_status() == binding.OK
+    ctx.selftest_wait_expiry(2_000_000)                  # about a millisecond of SM cycles
+    assert ctx.poll_device_status() == binding.ERR_TIMEOUT
+    assert ctx.poll_device_status() == binding.OK
+    scores = torch.rand(4096, device=cuda_device)
+    idx = torch.zeros(64, dtype=torch.int32, device=cuda_device)
+    ctx.select(scores, 64, 16, idx)                      # ordinary work still runs on the context
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == binding.OK
+    assert idx[-1].item() == 4095
+    ctx.close()
