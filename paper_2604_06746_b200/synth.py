@@ -54,6 +54,9 @@ class Workload:
     hub_span: Optional[int]       # contiguous active span length; None = use hub_layers
     hub_layers: Tuple[int, ...] = ()   # explicit active layers (used when hub_span is None)
     temperatures: Optional[Tuple[float, ...]] = None  # None = U[0.5, 2] per layer
+    temperature_draw: int = 0     # which draw of the temperature vector is used (earlier ones are
+                                  # discarded); fixed when a workload is designed so that no two
+                                  # layer transitions are nearly tied as the sharpest one
     sink: bool = False
     delimiters: bool = False
     heavy_tail: bool = False
@@ -134,7 +137,8 @@ def plan(wl: Workload) -> Plan:
     if wl.temperatures is not None:
         temps = np.asarray(wl.temperatures[:wl.n_layers], dtype=np.float64)
     else:
-        temps = rng.uniform(0.5, 2.0, size=wl.n_layers)
+        for _ in range(wl.temperature_draw + 1):
+            temps = rng.uniform(0.5, 2.0, size=wl.n_layers)
     return Plan(pos.astype(np.int64), active, temps)
 
 

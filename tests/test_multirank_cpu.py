@@ -48,3 +48,23 @@ def test_two_gloo_ranks_get_distinct_prompts_and_the_slowest_step_time():
     assert ms == 15.0                                                   # the maximum over ranks
     assert digests[0][0] != digests[1][0] and digests[0][1] != digests[1][1]   # different seeds, different data
     assert np.isclose(value, 2 * 2048 / 15e-3)                          # whole-job tokens per second
+
+
+def test_bare_launch_with_gpus_2_starts_two_ranks():
+    """`python bench.py --gpus 2` without a launcher must start its two ranks itself; the rank
+    plumbing is exercised on host memory (gloo) and rank 0 prints the job-level line."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--plumbing-check"],
+                         capture_output=True, text=True, timeout=300, env=env, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                              # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 15.0
+    assert line["prompts"][0][0] != line["prompts"][1][0] and line["prompts"][0][1] != line["prompts"][1][1]
+    assert np.isclose(line["value"], 2 * 2048 / 15e-3)
