@@ -232,6 +232,46 @@ def mass_recovery(scores: np.ndarray, idx: np.ndarray) -> float:
     return float(scores[np.asarray(idx, dtype=np.int64)].sum() / scores.sum())
 
 
+# ------------------------------------- Eq. 11 - 13 past the pivot (Algorithm 1, l > L*)
+def reduced_layer(q_win: np.ndarray, k: np.ndarray, scale: float, i_struct: np.ndarray,
+                  positions: np.ndarray, kv_budget: int, window: int) -> Dict[str, np.ndarray]:
+    """One layer past the pivot.  The sequence has been cut to the structural set (Eq. 11), so
+    the layer only has the keys ``k[:, i_struct]``; the window is the tail of ``i_struct`` (R9),
+    hence the window queries are unchanged and causality in reduced order is causality in
+    original order.  Scoring (Eq. 1 - 2) and selection (Eq. 13) run on that reduced sequence;
+    a selected reduced index ``r`` names the token whose original position is
+    ``positions[i_struct][r]`` (Eq. 12: the position ids travel with the tokens).
+
+    Returns ``S`` (reduced order), ``i_reduced`` (indices into the reduced sequence) and
+    ``i_kv`` (the same tokens as original position ids)."""
+    i_struct = np.asarray(i_struct, dtype=np.int64)
+    pos_reduced = np.asarray(positions)[i_struct]                       # P' = P[I_struct]
+    k_reduced = np.asarray(k, dtype=np.float64)[:, i_struct]
+    out = score_layer(q_win, k_reduced, scale)
+    i_reduced = select(out["S"], kv_budget, window)
+    return {"S": out["S"], "entropy": out["entropy"], "i_reduced": i_reduced, "i_kv": pos_reduced[i_reduced]}
+
+
+def prefill_reduced(layers: Sequence[Tuple[np.ndarray, np.ndarray, float]], positions: np.ndarray,
+                    window: int, kv_budget: int, struct_budget: int, lam: float = PAPER_LAMBDA,
+                    weights: Sequence[float] = PAPER_WEIGHTS, n_detect: Optional[int] = None,
+                    l_limit: Optional[int] = None) -> Dict[str, object]:
+    """Algorithm 1 with its truncation: the first ``n_detect`` layers (default: all) are scored on
+    the full sequence and give the pivot, the centrality at the pivot and ``I_struct``; every
+    layer ``l > L*`` then runs on the reduced sequence (``reduced_layer``).  ``recovery[l]`` is
+    the share of layer ``l``'s full-sequence attention that the structural set covers (Section
+    4.4, fidelity of hidden states), available here because the synthetic K is complete."""
+    n_detect = len(layers) if n_detect is None else n_detect
+    head = prefill(layers[:n_detect], window, kv_budget, struct_budget, lam, weights, l_limit)
+    L_star, i_struct = head["pivot"], head["i_struct"]
+    past, recovery = {}, {}
+    for l in range(L_star + 1, len(layers)):
+        q, k, sc = layers[l]
+        past[l] = reduced_layer(q, k, sc, i_struct, positions, kv_budget, window)
+        recovery[l] = mass_recovery(score_layer(q, k, sc)["S"], i_struct)
+    return {"head": head, "pivot": L_star, "i_struct": i_struct, "past": past, "recovery": recovery}
+
+
 # ------------------------------------------------------------------- Algorithm 1
 def prefill(layers: Sequence[Tuple[np.ndarray, np.ndarray, float]], window: int,
             kv_budget: int, struct_budget: int, lam: float = PAPER_LAMBDA,

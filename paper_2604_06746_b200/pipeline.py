@@ -83,6 +83,36 @@ class Prefill:
         self.ctx.compact(hidden[None], self.i_struct, self.hidden_out[None])
         self.ctx.compact(positions[None, :, None], self.i_struct, self.pos_out[None, :, None])
 
+    # -- Algorithm 1 past the pivot (Eq. 11-13 on the reduced sequence)
+    def enable_reduced(self) -> None:
+        """Buffers for layers scored after the truncation: K gathered at I_struct, the saliency of
+        the reduced sequence, its selection, and that selection as original position ids."""
+        dev, f32, i32 = self.device, torch.float32, torch.int32
+        nr = self.struct_budget
+        self.k_red = torch.empty((self.Hkv, nr, self.d), dtype=self.dtype, device=dev)
+        self.s_red = torch.zeros((self.L, nr), dtype=f32, device=dev)
+        self.metrics_red = torch.zeros((self.L, 3), dtype=f32, device=dev)
+        self.i_red = torch.zeros((self.L, self.kv_budget), dtype=i32, device=dev)
+        self.i_kv_pos = torch.zeros((self.L, self.kv_budget), dtype=i32, device=dev)
+        self.recovery = torch.zeros((self.L,), dtype=f32, device=dev)
+
+    def score_reduced(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, scale: float) -> None:
+        """Layer ``layer`` > L* on the keys that survived the truncation: gather K at I_struct
+        (Eq. 11), score the reduced sequence (the window is its tail, so the queries are unchanged)."""
+        self.ctx.compact(k, self.i_struct, self.k_red)
+        self.ctx.score_layer(q_win, self.k_red, scale, self.s_red[layer], self.metrics_red[layer],
+                             flags=self.flags)
+
+    def select_reduced(self, first: int, last: int) -> None:
+        """Eq. 13 on the reduced sequences of layers ``first .. last - 1`` (one batched launch), then
+        each index list mapped back to original positions through the gathered position ids
+        (Eq. 12; ``compact_hidden`` must have filled ``pos_out``)."""
+        if last <= first:
+            return
+        self.ctx.select(self.s_red[first:last], self.kv_budget, self.w, self.i_red[first:last])
+        for l in range(first, last):
+            self.ctx.compact(self.pos_out[None, :, None], self.i_red[l], self.i_kv_pos[l][None, :, None])
+
     def run(self, layers: Sequence[Dict[str, torch.Tensor]], hidden: Optional[torch.Tensor] = None,
             positions: Optional[torch.Tensor] = None) -> int:
         """Whole path over resident per-layer tensors (dicts with q_win, k, v, scale)."""
