@@ -95,7 +95,7 @@ WORKLOADS: Dict[str, Workload] = {
                      hub_layers=(1, 2), temperatures=(0.5, 1.0, 2.0, 1.0), sink=True),
     "llama32k": Workload("llama32k", 1, 32, 32, 8, 128, 32768, 64, (2048,), "bf16", 64, 8),
     "llama128k": Workload("llama128k", 2, 32, 32, 8, 128, 131072, 64, (1024, 4096, 16384), "bf16",
-                          256, 8, sink=True, delimiters=True),
+                          256, 8, sink=True, delimiters=True, temperature_draw=11),
     "qwen64k": Workload("qwen64k", 3, 28, 28, 4, 128, 65536, 128, (4096,), "bf16", 128, 8,
                         heavy_tail=True),
     "llama256k": Workload("llama256k", 4, 32, 32, 8, 128, 262144, 64, (8192,), "bf16", 256, 8,

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("name,seq,layers,budget,n_detect", [
     ("llama32k", 6000 + 13, 6, 300, 4),      # reduced length 600: ragged last key tile
     ("qwen64k", 5000, 6, 700, 4),            # GQA 7, window 128, reduced length 1400
-    ("llama128k", 20000, 8, 1024, 6),        # sink + delimiters, reduced length 2048
+    ("llama128k", 20000, 9, 1024, 6),        # sink + delimiters, reduced length 2048
 ])
 def test_post_pivot_flow_matches_the_oracle(cuda_device, name, seq, layers, budget, n_detect):
     from paper_2604_06746_b200 import binding, pipeline
