@@ -294,3 +294,26 @@ def prefill(layers: Sequence[Tuple[np.ndarray, np.ndarray, float]], window: int,
         "i_struct": select(C, struct_budget, window),
         "i_kv": np.stack([select(s_hist[l], kv_budget, window) for l in range(len(outs))]),
     }
+
+
+# --------------------------- Section 4.1 (implementation details): batches of prompts
+def prefill_batch(prompts: Sequence[Sequence[Tuple[np.ndarray, np.ndarray, float]]], window: int,
+                  kv_budgets: Sequence[int], struct_budgets: Sequence[int], lam: float = PAPER_LAMBDA,
+                  weights: Sequence[float] = PAPER_WEIGHTS,
+                  l_limit: Optional[int] = None) -> Dict[str, object]:
+    """A batch of prompts of different lengths: every prompt is an independent problem with its
+    own length, pivot and index sets (``prefill`` per prompt).  ``reduced_at[b, l]`` is the
+    masked state transition: True where layer ``l`` of prompt ``b`` runs past that prompt's pivot,
+    i.e. on its reduced sequence.  Index lists come back padded with -1 to the largest budget
+    (the padded addressing of a batch); padding is never a token."""
+    per = [prefill(layers, window, kb, sb, lam, weights, l_limit)
+           for layers, kb, sb in zip(prompts, kv_budgets, struct_budgets)]
+    L = max(len(p) for p in prompts)
+    pivots = np.array([r["pivot"] for r in per], dtype=np.int64)
+    reduced_at = np.arange(L)[None, :] > pivots[:, None]
+    i_struct = np.full((len(per), max(struct_budgets)), -1, dtype=np.int64)
+    i_kv = np.full((len(per), L, max(kv_budgets)), -1, dtype=np.int64)
+    for b, r in enumerate(per):
+        i_struct[b, :struct_budgets[b]] = r["i_struct"]
+        i_kv[b, :len(prompts[b]), :kv_budgets[b]] = r["i_kv"]
+    return {"per_prompt": per, "pivots": pivots, "reduced_at": reduced_at, "i_struct": i_struct, "i_kv": i_kv}
