@@ -188,6 +188,7 @@ class Resident:
         if timed: e[0].record()
         for l, t in enumerate(layers):
             pf.score(l, t["q_win"], t["k"], t["scale"])
+        pf.finish_scores(len(layers))          # Eq. 5-6 of all layers (batched): part of the scoring phase
         if timed: e[1].record()
         pf.detect_and_select(len(layers))
         if timed: e[2].record()
@@ -256,6 +257,12 @@ def time_streamed(wl, pl, kv_budget, dev, sweeps=2):
             del t
         a, b = ev(), ev()
         a.record()
+        pf.finish_scores(wl.n_layers)
+        b.record()
+        torch.cuda.synchronize()
+        acc["score"] += a.elapsed_time(b)
+        a, b = ev(), ev()
+        a.record()
         pf.detect_and_select(wl.n_layers)
         b.record()
         torch.cuda.synchronize()
@@ -321,10 +328,12 @@ def compaction_figures(wl, kv_budget, compact_ms_per_step, peaks):
 
 def launches_per_step(wl, flags):
     from paper_2604_06746_b200 import binding
-    per_layer = 5 if not (flags & binding.FLAG_NO_HEAD_STATS) else 4
-    if wl.dtype != "bf16":
-        per_layer += 1
-    return wl.n_layers * per_layer + 1 + 2 + wl.n_layers + 2
+    # per layer: scorer pass 1, pass 2, column reduce + metrics (the CUDA-core scorer adds a row
+    # finalisation); per step: batched head statistics (2), accumulate, 2 selections, one K/V gather
+    # per layer, hidden states, positions
+    per_layer = 3 if wl.dtype == "bf16" else 4
+    stats = 0 if (flags & binding.FLAG_NO_HEAD_STATS) else 2
+    return wl.n_layers * per_layer + stats + 1 + 2 + wl.n_layers + 2
 
 
 # ------------------------------------------------------------------------------------------------

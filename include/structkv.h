@@ -116,6 +116,26 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
                                      void* stream);
 
 /*
+ * Eq. 5 and Eq. 6 (Section 3.3) for several layers at once, from the pooled per-head attention
+ * that structkv_score_layer wrote to head_cols_out.  A caller that scores many layers passes
+ * STRUCTKV_FLAG_NO_HEAD_STATS and a distinct head_cols_out slab per layer, then makes ONE call
+ * here before the pivot: the per-head selections of all layers run side by side instead of as
+ * a chain of short dependent launches after every layer.
+ *
+ *   head_cols     device, fp32: entry (l, h, j) at head_cols + l*layer_stride + h*col_stride + j,
+ *                 each (l, h) vector non-negative and summing to 1 (Eq. 2's per-head pooling).
+ *   n_layers      1 .. 128.
+ *   n             N, the number of keys of every vector; col_stride >= n.
+ *   metrics       device, [n_layers, 3] fp32: entries [l][1] (sparsity) and [l][2] (variance) are
+ *                 written, [l][0] (entropy) is left untouched.
+ * Results equal those of structkv_score_layer without the flag.  Uses the context's workspace
+ * (calls on one context are ordered by the caller).  Errors: INVALID_ARG, CUDA.  Asynchronous.
+ */
+structkv_status structkv_head_stats(structkv_ctx* ctx, const float* head_cols, long long layer_stride,
+                                    long long col_stride, int n_layers, int n, float* metrics,
+                                    void* stream);
+
+/*
  * structkv_score_layer without a context and without a caller workspace.  The paper has no
  * counterpart: this entry point exists for integration only.
  *

@@ -52,6 +52,8 @@ lib.structkv_score_layer_static.restype = _i
 lib.structkv_score_layer_static.argtypes = [ctypes.POINTER(Config), _vp, _vp, _ll, _ll, _i, _f, _f, _vp, _vp,
                                             _vp, _vp, _u, _vp]
 STATIC_SCRATCH_BYTES = 8 << 20
+lib.structkv_head_stats.restype = _i
+lib.structkv_head_stats.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _vp, _vp]
 lib.structkv_pivot.restype = _i
 lib.structkv_pivot.argtypes = [_vp, _vp, _i, ctypes.POINTER(_f), _i, ctypes.POINTER(_i),
                                ctypes.POINTER(_f), _vp]
@@ -168,6 +170,15 @@ class Context:
                                         k.shape[1], scale, lam, s_out.data_ptr(), _ptr(c_inout),
                                         _ptr(head_cols_out), metrics_out.data_ptr(), flags,
                                         _stream(stream)), "structkv_score_layer")
+
+    def head_stats(self, head_cols: torch.Tensor, metrics: torch.Tensor,
+                   stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_head_stats: ``head_cols [n_layers, H, n]`` -> ``metrics [n_layers, 3]`` columns 1 and 2."""
+        assert head_cols.dim() == 3 and head_cols.stride(2) == 1 and head_cols.dtype == torch.float32
+        assert metrics.is_contiguous() and metrics.shape == (head_cols.shape[0], 3)
+        _check(lib.structkv_head_stats(self._h, head_cols.data_ptr(), head_cols.stride(0), head_cols.stride(1),
+                                       head_cols.shape[0], head_cols.shape[2], metrics.data_ptr(),
+                                       _stream(stream)), "structkv_head_stats")
 
     def pivot(self, metrics: torch.Tensor, weights: Sequence[float] = (0.2, 0.3, 0.5), l_limit: int = -1,
               stream: Optional[torch.cuda.Stream] = None) -> Tuple[int, list]:

@@ -48,7 +48,7 @@ Workspace carve_workspace(const structkv_config& cfg, void* base) {
   w.row_lse2 = (float*)take(rows_pad * sizeof(float));
   w.row_ent = (float*)take(rows_pad * sizeof(float));
   w.cols = (float*)take((size_t)cfg.n_q_heads * n_pad * sizeof(float));
-  w.head_part = (float*)take((size_t)cfg.n_q_heads * 4 * sizeof(float));
+  w.head_part = (float*)take((size_t)kMaxStatLayers * cfg.n_q_heads * 4 * sizeof(float));
   w.bytes = off;
   return w;
 }
@@ -155,10 +155,19 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   }
   e = use_tc ? launch_score_tc(c, a, &parts, 2, st) : launch_score_simt(c, a, &parts, 2, st);
   if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
-  e = launch_reduce_columns(c, a.cols, a.col_stride, n_keys, lambda, s_out, c_inout, st);
-  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
-  e = launch_metrics(c, a.cols, a.col_stride, n_keys, !(flags & STRUCTKV_FLAG_NO_HEAD_STATS), metrics_out, st);
+  e = launch_reduce_finish(c, a.cols, a.col_stride, n_keys, lambda, s_out, c_inout,
+                           !(flags & STRUCTKV_FLAG_NO_HEAD_STATS), metrics_out, st);
   return e == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
+}
+
+structkv_status structkv_head_stats(structkv_ctx* ctx, const float* head_cols, long long layer_stride,
+                                    long long col_stride, int n_layers, int n, float* metrics,
+                                    void* stream) {
+  if (!ctx || !head_cols || !metrics) return STRUCTKV_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > kMaxStatLayers || n < 1 || col_stride < n) return STRUCTKV_ERR_INVALID_ARG;
+  if (n_layers > 1 && layer_stride < (long long)ctx->c.cfg.n_q_heads * col_stride) return STRUCTKV_ERR_INVALID_ARG;
+  return launch_head_stats_batch(ctx->c, head_cols, layer_stride, col_stride, n_layers, n, metrics,
+                                 (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
 }
 
 structkv_status structkv_pivot(structkv_ctx* ctx, const float* metrics_dev, int n_layers,

@@ -12,6 +12,7 @@ namespace skv {
 constexpr int kKeyTile = 128;        // keys per tile in every scorer
 constexpr int kMaxParts = 160;       // upper bound on key segments per score row
 constexpr int kRowBlock = 256;       // score rows (head, window row) per tensor-core row block
+constexpr int kMaxStatLayers = 128;  // layers one batched head-statistics call may cover
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -22,7 +23,7 @@ struct Workspace {
   float* row_lse2;      // [rows_pad] log2-domain log-sum-exp of each score row
   float* row_ent;       // [rows_pad] entropy of each score row (nats)
   float* cols;          // [H][n_pad] pooled per-head attention when the caller passes none
-  float* head_part;     // [H][4] per-head {sum of squared deviations from 1/n, top-k mass}
+  float* head_part;     // [kMaxStatLayers][H][4] per-(layer, head) {sum of squared deviations from 1/n, top-k mass}
   size_t bytes;
 };
 
@@ -71,14 +72,16 @@ cudaError_t launch_wait_probe(unsigned long long limit_cycles, int* status, cuda
 // CUDA-core scorer; the tensor-core scorer does this at the start of its second pass).
 cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st);
 
-// S_j = sum_h cols[h][j]; optional C <- lambda C + S.
-cudaError_t launch_reduce_columns(const Ctx& ctx, const float* cols, long long col_stride, int n,
-                                  float lambda, float* s_out, float* c_inout, cudaStream_t st);
+// S_j = sum_h cols[h][j]; optional C <- lambda C + S; then the layer's metrics: metrics[0] from
+// row_ent (Eq. 4); metrics[1..2] from the pooled per-head attention (Eq. 5-6, computed here when
+// with_head_stats), or NaN.
+cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long col_stride, int n, float lambda,
+                                 float* s_out, float* c_inout, bool with_head_stats, float* metrics,
+                                 cudaStream_t st);
 
-// metrics[0] from row_ent (Eq. 4); metrics[1..2] from the pooled per-head attention (Eq. 5-6),
-// or NaN when head statistics are disabled.
-cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stride, int n,
-                           bool with_head_stats, float* metrics, cudaStream_t st);
+// Eq. 5-6 for n_layers layers at once from their pooled per-head attention: writes metrics[l][1..2].
+cudaError_t launch_head_stats_batch(const Ctx& ctx, const float* cols, long long layer_stride, long long col_stride,
+                                    int n_layers, int n, float* metrics, cudaStream_t st);
 
 cudaError_t launch_accumulate(const float* s_hist, long long row_stride, int pivot, int n,
                               float lambda, float* c_out, cudaStream_t st);

@@ -10,8 +10,6 @@ namespace cg = cooperative_groups;
 namespace skv {
 namespace {
 
-constexpr int kFinalThreads = 1024;
-
 __device__ __forceinline__ float block_sum_1024(float v, float* red) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -69,17 +67,64 @@ finalize_rows(const float4* __restrict__ row_part, int parts, int rows_pad, int 
 }
 
 // S_j = sum over heads (fixed order) of cols[h][j];  C_j <- lambda C_j + S_j  (Eq. 2, Eq. 3).
-__global__ void reduce_columns(const float* __restrict__ cols, long long col_stride, int H, int n,
-                               float lambda, float* __restrict__ s_out,
-                               float* __restrict__ c_inout) {
+// Four keys per thread where the layout allows 16-byte accesses.  Block 0 also finishes the
+// layer's metrics: metrics[0] = mean entropy of the valid score rows (Eq. 4); metrics[1] = mean
+// over heads of the top-mass (Eq. 5), metrics[2] = mean over heads of (sum of squared deviations
+// from 1/n) / n (Eq. 6), both from head_part, or NaN when head statistics are not computed here.
+// Fixed summation order throughout.
+constexpr int kRcThreads = 256;
+template <int VEC>
+__global__ void __launch_bounds__(kRcThreads)
+reduce_finish(const float* __restrict__ cols, long long col_stride, int H, int n, float lambda,
+              float* __restrict__ s_out, float* __restrict__ c_inout, const float* __restrict__ row_ent,
+              int rows_pad, int rows_pg_pad, int rows_pg, int n_valid, const float* __restrict__ head_part,
+              int with_head_stats, float* __restrict__ metrics) {
+  __shared__ float red[33];
   pdl_trigger();
   pdl_wait();
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= n) return;
-  float s = 0.f;
-  for (int h = 0; h < H; ++h) s += cols[(size_t)h * col_stride + j];
-  s_out[j] = s;
-  if (c_inout) c_inout[j] = fmaf(lambda, c_inout[j], s);
+  const int j = (blockIdx.x * kRcThreads + threadIdx.x) * VEC;
+  if (VEC == 4) {
+    if (j < n) {                                   // n is a multiple of 4 in this instantiation
+      float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+      for (int h = 0; h < H; ++h) {
+        const float4 v = *reinterpret_cast<const float4*>(cols + (size_t)h * col_stride + j);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      }
+      *reinterpret_cast<float4*>(s_out + j) = s;
+      if (c_inout) {
+        float4 c = *reinterpret_cast<const float4*>(c_inout + j);
+        c.x = fmaf(lambda, c.x, s.x); c.y = fmaf(lambda, c.y, s.y);
+        c.z = fmaf(lambda, c.z, s.z); c.w = fmaf(lambda, c.w, s.w);
+        *reinterpret_cast<float4*>(c_inout + j) = c;
+      }
+    }
+  } else if (j < n) {
+    float s = 0.f;
+    for (int h = 0; h < H; ++h) s += cols[(size_t)h * col_stride + j];
+    s_out[j] = s;
+    if (c_inout) c_inout[j] = fmaf(lambda, c_inout[j], s);
+  }
+  if (blockIdx.x != 0) return;
+  float ent = 0.f;
+  for (int r = threadIdx.x; r < rows_pad; r += kRcThreads)
+    if ((r % rows_pg_pad) < rows_pg) ent += row_ent[r];
+  const float tot = block_sum_1024(ent, red);
+  if (threadIdx.x != 0) return;
+  metrics[0] = tot / (float)n_valid;
+  if (!with_head_stats) {
+    metrics[1] = __int_as_float(0x7fc00000);
+    metrics[2] = __int_as_float(0x7fc00000);
+    return;
+  }
+  float rho = 0.f, var = 0.f;
+  const float inv_n = 1.f / (float)n;
+  for (int h = 0; h < H; ++h) {
+    rho += head_part[h * 4 + 1];
+    var += head_part[h * 4 + 0] * inv_n;
+  }
+  metrics[1] = rho / (float)H;
+  metrics[2] = var / (float)H;
 }
 
 // Per head: sum of squared deviations from 1/n (Eq. 6: the pooled vector sums to 1, so 1/n is its
@@ -102,8 +147,8 @@ constexpr int kHsItems = 16;      // entries per thread kept in registers betwee
 
 // Shared memory of head_stats: hist[kHsBins][kHsCopies] | merged[2][kHsBins] (dynamic, 80 KB).
 __global__ void __cluster_dims__(kHsCluster, 1, 1) __launch_bounds__(kHsThreads)
-head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rho,
-           float* __restrict__ head_part) {
+head_stats(const float* __restrict__ cols, long long layer_stride, long long col_stride, int H, int n,
+           int k_rho, float* __restrict__ head_part) {
   extern __shared__ unsigned hs_smem[];
   unsigned* hist = hs_smem;                          // this CTA's counts, kHsCopies per bin
   unsigned* merged = hs_smem + kHsBins * kHsCopies;  // cluster-wide counts of the two levels (CTA 0's copy counts)
@@ -113,8 +158,8 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   __shared__ unsigned sel_bin, sel_rem;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
-  const int head = blockIdx.x / kHsCluster;
-  const float* a = cols + (size_t)head * col_stride;
+  const int head = blockIdx.x / kHsCluster;          // (layer, head) pair: one cluster each
+  const float* a = cols + (size_t)(head / H) * layer_stride + (size_t)(head % H) * col_stride;
   const int tid = threadIdx.x, copy = tid & (kHsCopies - 1);
   const int per = (n + kHsCluster - 1) / kHsCluster;
   const int lo = rank * per, hi = min(n, lo + per);
@@ -216,35 +261,21 @@ head_stats(const float* __restrict__ cols, long long col_stride, int n, int k_rh
   }
 }
 
-// metrics[0] = mean entropy of the valid score rows (Eq. 4);  metrics[1] = mean_h top-mass
-// (Eq. 5);  metrics[2] = mean_h (sum of squared deviations from 1/n) / n (Eq. 6).  With head
-// statistics disabled metrics[1..2] are NaN.  One block, fixed summation order.
-__global__ void __launch_bounds__(kFinalThreads)
-finish_metrics(const float* __restrict__ row_ent, int rows_pad, int rows_pg_pad, int rows_pg,
-               int n_valid, const float* __restrict__ head_part, int H, int n, int with_head_stats,
-               float* __restrict__ metrics) {
-  __shared__ float red[33];
+// Eq. 5-6 of a batch of layers from their per-head parts: one thread per layer.
+__global__ void head_metrics(const float* __restrict__ head_part, int n_layers, int H, int n,
+                             float* __restrict__ metrics) {
   pdl_trigger();
   pdl_wait();
-  float ent = 0.f;
-  for (int r = threadIdx.x; r < rows_pad; r += kFinalThreads)
-    if ((r % rows_pg_pad) < rows_pg) ent += row_ent[r];
-  const float tot = block_sum_1024(ent, red);
-  if (threadIdx.x != 0) return;
-  metrics[0] = tot / (float)n_valid;
-  if (!with_head_stats) {
-    metrics[1] = __int_as_float(0x7fc00000);
-    metrics[2] = __int_as_float(0x7fc00000);
-    return;
-  }
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= n_layers) return;
   float rho = 0.f, var = 0.f;
   const float inv_n = 1.f / (float)n;
   for (int h = 0; h < H; ++h) {
-    rho += head_part[h * 4 + 1];
-    var += head_part[h * 4 + 0] * inv_n;
+    rho += head_part[((size_t)l * H + h) * 4 + 1];
+    var += head_part[((size_t)l * H + h) * 4 + 0] * inv_n;
   }
-  metrics[1] = rho / (float)H;
-  metrics[2] = var / (float)H;
+  metrics[l * 3 + 1] = rho / (float)H;
+  metrics[l * 3 + 2] = var / (float)H;
 }
 
 // c_out[j] = sum_{l <= pivot} lambda^(pivot - l) s_hist[l][j], as the recursion c = lambda c + s.
@@ -268,29 +299,47 @@ cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_reduce_columns(const Ctx& ctx, const float* cols, long long col_stride, int n,
-                                  float lambda, float* s_out, float* c_inout, cudaStream_t st) {
-  return launch_pdl(reduce_columns, dim3((n + 255) / 256), dim3(256), 0, st, cols, col_stride,
-                    ctx.cfg.n_q_heads, n, lambda, s_out, c_inout);
+static cudaError_t launch_head_stats(const float* cols, long long layer_stride, long long col_stride, int n_layers,
+                                     int H, int n, float* head_part, cudaStream_t st) {
+  int k_rho = n / 10;
+  if (k_rho < 1) k_rho = 1;
+  const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
+  cudaError_t e = cudaFuncSetAttribute(head_stats, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(head_stats, dim3(n_layers * H * kHsCluster), dim3(kHsThreads), smem, st, cols, layer_stride,
+                    col_stride, H, n, k_rho, head_part);
 }
 
-cudaError_t launch_metrics(const Ctx& ctx, const float* cols, long long col_stride, int n,
-                           bool with_head_stats, float* metrics, cudaStream_t st) {
+cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long col_stride, int n, float lambda,
+                                 float* s_out, float* c_inout, bool with_head_stats, float* metrics,
+                                 cudaStream_t st) {
+  const int H = ctx.cfg.n_q_heads;
   if (with_head_stats) {
-    int k_rho = n / 10;
-    if (k_rho < 1) k_rho = 1;
-    const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
-    cudaError_t e = cudaFuncSetAttribute(head_stats, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(head_stats, dim3(ctx.cfg.n_q_heads * kHsCluster), dim3(kHsThreads), smem, st, cols,
-                   col_stride, n, k_rho, ctx.ws.head_part);
+    const cudaError_t e = launch_head_stats(cols, 0, col_stride, 1, H, n, ctx.ws.head_part, st);
     if (e != cudaSuccess) return e;
   }
   const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
-  const int rows_pg = (ctx.cfg.n_q_heads / ctx.cfg.n_kv_heads) * ctx.cfg.window;
-  return launch_pdl(finish_metrics, dim3(1), dim3(kFinalThreads), 0, st, (const float*)ctx.ws.row_ent,
-                    ctx.rows_pad, rows_pg_pad, rows_pg, ctx.rows, (const float*)ctx.ws.head_part,
-                    ctx.cfg.n_q_heads, n, with_head_stats ? 1 : 0, metrics);
+  const int rows_pg = (H / ctx.cfg.n_kv_heads) * ctx.cfg.window;
+  const bool vec = n % 4 == 0 && col_stride % 4 == 0 && ((uintptr_t)cols % 16) == 0 &&
+                   ((uintptr_t)s_out % 16) == 0 && ((uintptr_t)c_inout % 16) == 0;
+  if (vec)
+    return launch_pdl(reduce_finish<4>, dim3((n / 4 + kRcThreads - 1) / kRcThreads), dim3(kRcThreads), 0, st, cols,
+                      col_stride, H, n, lambda, s_out, c_inout, (const float*)ctx.ws.row_ent, ctx.rows_pad,
+                      rows_pg_pad, rows_pg, ctx.rows, (const float*)ctx.ws.head_part, with_head_stats ? 1 : 0,
+                      metrics);
+  return launch_pdl(reduce_finish<1>, dim3((n + kRcThreads - 1) / kRcThreads), dim3(kRcThreads), 0, st, cols,
+                    col_stride, H, n, lambda, s_out, c_inout, (const float*)ctx.ws.row_ent, ctx.rows_pad,
+                    rows_pg_pad, rows_pg, ctx.rows, (const float*)ctx.ws.head_part, with_head_stats ? 1 : 0,
+                    metrics);
+}
+
+cudaError_t launch_head_stats_batch(const Ctx& ctx, const float* cols, long long layer_stride, long long col_stride,
+                                    int n_layers, int n, float* metrics, cudaStream_t st) {
+  const int H = ctx.cfg.n_q_heads;
+  cudaError_t e = launch_head_stats(cols, layer_stride, col_stride, n_layers, H, n, ctx.ws.head_part, st);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(head_metrics, dim3((n_layers + 63) / 64), dim3(64), 0, st, (const float*)ctx.ws.head_part,
+                    n_layers, H, n, metrics);
 }
 
 cudaError_t launch_accumulate(const float* s_hist, long long row_stride, int pivot, int n,

@@ -37,6 +37,8 @@ constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 
 struct TcParams {
   int n_keys, window, group, rows_pg, rows_pg_pad, rows_pad, n_rb, segs, n_tiles, n_pairs;
   float c2;                            // scale * log2(e)
+  float inv_c2;                        // 1 / c2, or 0 when the fold of -lse into the MMA is off
+  int fold;                            // pass 2: the accumulator already holds q.k - lse / c2
   float4* row_part;                    // pass 1 out, pass 2 in: [segs][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride]
@@ -69,6 +71,33 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
+}
+// Same test, letting the hardware suspend the thread for up to `ns` nanoseconds while the phase
+// is incomplete: a waiting producer then issues (almost) no instructions on its scheduler.
+#ifndef SKV_WAIT_HINT_NS
+#define SKV_WAIT_HINT_NS 1000
+#endif
+__device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"((uint32_t)SKV_WAIT_HINT_NS) : "memory");
+  return ok != 0;
+}
+// Bounded wait of a producer (TMA / MMA warp): long, rarely latency critical.
+__device__ __forceinline__ bool mbar_wait_producer(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                   unsigned long long limit) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (SKV_WAIT_HINT_NS > 0 ? mbar_try_suspend(bar, parity) : mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return false; }
+  }
 }
 // Bounded wait.  Returns false if the barrier did not flip within `limit` cycles or the CTA is
 // aborting; the first waiter whose bound expires raises the CTA's abort flag.
@@ -197,7 +226,7 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
   return pack2(fast_exp2(x0), fast_exp2(x1));
 }
 // Scalar form of the same polynomial (pass 1).
-__device__ __forceinline__ float exp2_poly1(float x) {
+[[maybe_unused]] __device__ __forceinline__ float exp2_poly1(float x) {
   x = fminf(fmaxf(x, -125.f), 126.f);
   const float t = x + 12582912.0f;
   const float f = x - (t - 12582912.0f);
@@ -206,9 +235,17 @@ __device__ __forceinline__ float exp2_poly1(float x) {
   p = fmaf(p, f, 0.9999280572f);
   return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
-// In pass 1, of every 8 consecutive elements the first kPoly1 take the polynomial.
+// In pass 1, of every 8 consecutive elements (element pairs in the packed form) the first kPoly1
+// take the polynomial.
 #ifndef SKV_POLY1
-#define SKV_POLY1 2
+#define SKV_POLY1 0
+#endif
+#ifndef SKV_PACK1
+#define SKV_PACK1 0
+#endif
+// Pass 2: subtract lse inside the MMA (one extra K-step) instead of loading it from shared memory.
+#ifndef SKV_FOLD
+#define SKV_FOLD 0
 #endif
 constexpr int kPoly1 = SKV_POLY1;
 // In pass 2, of every 8 consecutive element pairs the first kPoly2 take the polynomial, the
@@ -228,6 +265,21 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
   d |= (uint64_t)2 << 61;                          // 128-byte swizzle
   return d;
+}
+// Shared-memory matrix descriptor of an unswizzled K-major operand of 16 columns (one MMA
+// K-step): 8-row x 16-byte core matrices of 128 contiguous bytes, the two K halves of a row
+// group 128 bytes apart, row groups 256 bytes apart.  Element (row, k) therefore sits at
+// (row / 8) * 256 + (k / 8) * 128 + (row % 8) * 16 + (k % 8) * 2.
+__device__ __forceinline__ uint64_t smem_desc_k16(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3fffu);
+  d |= (uint64_t)(128 >> 4) << 16;                 // between the core matrices of one row group (K direction)
+  d |= (uint64_t)(256 >> 4) << 32;                 // between row groups
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+__device__ __forceinline__ uint32_t k16_offset(int row, int k) {
+  return (uint32_t)((row >> 3) * 256 + (k >> 3) * 128 + (row & 7) * 16 + (k & 7) * 2);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, tile M x N.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N) {
@@ -257,7 +309,7 @@ struct Smem {
 // Barrier slots (8 bytes each) inside the barrier area.
 enum { kBarFull = 0, kBarEmpty = kStages, kBarQ = 2 * kStages, kBarAccFull = 2 * kStages + 1,
        kBarAccEmpty = kBarAccFull + kAccStages, kBarDrain = kBarAccEmpty + kAccStages,
-       kBarCount = kBarDrain + 1 };
+       kBarExt = kBarDrain + 1, kBarCount = kBarExt + 1 };
 
 template <int D, int PASS, int W>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -296,6 +348,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       mbar_init(bars + 8 * (kBarAccEmpty + a), kComputeWarps);   // one arrival per compute warp
     }
     mbar_init(bars + 8 * kBarDrain, 1);
+    mbar_init(bars + 8 * kBarExt, 1);
     *abort_flag = 0;
     *mma_in_flight = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -328,7 +381,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       for (int t = 0; t < n_load; ++t) {
         const int s = t % kStages;
         const uint32_t ph = (uint32_t)(t / kStages) & 1u;
-        if (!mbar_wait(bars + 8 * (kBarEmpty + s), ph ^ 1u, abort_flag)) break;
+        if (!mbar_wait_producer(bars + 8 * (kBarEmpty + s), ph ^ 1u, abort_flag, kWaitCycles)) break;
         mbar_expect_tx(bars + 8 * (kBarFull + s), L::kKBytes);
         // a pair's second tile may lie wholly beyond the last key: TMA fills it with zeros and
         // the causal mask discards it
@@ -348,19 +401,19 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     if (lane == 0 && n_my > 0) {
       constexpr uint32_t idesc = instr_desc(128, 256);
       const uint64_t q_desc0 = smem_desc(base + L::kQOff), k_desc0 = smem_desc(base + L::kKOff);
-      bool ok = mbar_wait(bars + 8 * kBarQ, 0, abort_flag);
+      bool ok = mbar_wait_producer(bars + 8 * kBarQ, 0, abort_flag, kWaitCycles);
       // descriptors differ only in the start-address field (16-byte units, no carry out of it)
       if (PASS == 1) {
         // unit u = (pair, row half): A = one 128-row half of Q, B = the pair's 256 keys
         for (int t = 0, u = 0; ok && t < n_my; ++t) {
           const int s0 = (2 * t) % kStages;
           const uint32_t ph = (uint32_t)((2 * t) / kStages) & 1u;
-          if (!mbar_wait(bars + 8 * (kBarFull + s0), ph, abort_flag)) break;
-          if (!mbar_wait(bars + 8 * (kBarFull + s0 + 1), ph, abort_flag)) break;
+          if (!mbar_wait_producer(bars + 8 * (kBarFull + s0), ph, abort_flag, kWaitCycles)) break;
+          if (!mbar_wait_producer(bars + 8 * (kBarFull + s0 + 1), ph, abort_flag, kWaitCycles)) break;
           const uint64_t kd = k_desc0 + (uint64_t)((s0 * L::kKSub) >> 4);
           for (int hf = 0; hf < n_half; ++hf, ++u) {
             const int a = u % kAccStages;
-            if (!mbar_wait(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(u / kAccStages) & 1u) ^ 1u, abort_flag)) {
+            if (!mbar_wait_producer(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(u / kAccStages) & 1u) ^ 1u, abort_flag, kWaitCycles)) {
               ok = false;
               break;
             }
@@ -381,8 +434,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       } else {
         for (int t = 0; ok && t < n_my; ++t) {
           const int s = t % kStages, a = t % kAccStages;
-          if (!mbar_wait(bars + 8 * (kBarFull + s), (uint32_t)(t / kStages) & 1u, abort_flag)) break;
-          if (!mbar_wait(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(t / kAccStages) & 1u) ^ 1u, abort_flag)) break;
+          if (!mbar_wait_producer(bars + 8 * (kBarFull + s), (uint32_t)(t / kStages) & 1u, abort_flag, kWaitCycles)) break;
+          if (!mbar_wait_producer(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(t / kAccStages) & 1u) ^ 1u, abort_flag, kWaitCycles)) break;
           tc_fence_after();
           const uint64_t kd = k_desc0 + (uint64_t)((s * L::kKSub) >> 4);
 #pragma unroll
@@ -392,6 +445,13 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
             tc_mma_bf16(tmem + a * 256, kd + (ko >> 4), q_desc0 + (qo >> 4), idesc, kk > 0);
           }
           *mma_in_flight = 1;
+          if (p.fold) {
+            // one more K-step adds -lse / c2 of every row: ones (key side) x three bf16 pieces of
+            // the value (row side), written by the compute warps once pass 1 has completed
+            if (t == 0 && !mbar_wait_producer(bars + 8 * kBarExt, 0, abort_flag, kWaitCycles)) break;
+            tc_mma_bf16(tmem + a * 256, smem_desc_k16(base + L::kMergeOff + 4096),
+                        smem_desc_k16(base + L::kMergeOff + 8192), idesc, 1);
+          }
           tc_commit(bars + 8 * (kBarEmpty + s));       // K stage reusable once these MMAs have read it
           tc_commit(bars + 8 * (kBarAccFull + a));     // accumulator ready for the compute warps
         }
@@ -434,6 +494,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       // the 64 keys [sub * 64, sub * 64 + 64) of every pair.
       struct RowStat { float ref, Z, U; };
       RowStat st[2] = {{-INFINITY, 0.f, 0.f}, {-INFINITY, 0.f, 0.f}};
+      const uint64_t c22 = pack2(p.c2, p.c2);
       const int row_lo = quarter * 32 + lane;
       const int i_win = row_lo % p.window;          // window row of this thread's rows (the window divides 128)
       const int t_pos = p.n_keys - p.window + i_win;                     // their position: they see keys <= t_pos
@@ -441,6 +502,30 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible;
       // of every 8 elements the first kPoly1 are exponentiated on the FMA pipe
       auto accumulate = [&](RowStat& r) {
+#if SKV_PACK1
+        // packed fp32: one instruction for two elements wherever the operation is not the exponential
+        const uint64_t nref2 = pack2(-r.ref, -r.ref);
+        uint64_t Z2 = pack2(r.Z, 0.f), U2 = pack2(r.U, 0.f);
+#pragma unroll
+        for (int pr = 0; pr < 16; ++pr) {
+          const uint64_t x2 = fma2(pack2(v[2 * pr], v[2 * pr + 1]), c22, nref2);
+          uint64_t p2;
+          if ((pr & 7) < kPoly1) {
+            float x0, x1;
+            unpack2(x2, x0, x1);
+            p2 = exp2_poly2(pack2(fminf(fmaxf(x0, -125.f), 126.f), fminf(fmaxf(x1, -125.f), 126.f)));
+          } else {
+            p2 = exp2_sfu2(x2);
+          }
+          Z2 = add2(Z2, p2);
+          U2 = fma2(p2, x2, U2);
+        }
+        float a, b;
+        unpack2(Z2, a, b);
+        r.Z = a + b;
+        unpack2(U2, a, b);
+        r.U = a + b;
+#else
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const float x = fmaf(v[e], p.c2, -r.ref);
@@ -448,6 +533,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
           r.Z += pr;
           r.U = fmaf(pr, x, r.U);
         }
+#endif
       };
       // same with the causal mask, moving the reference up to the chunk maximum first
       // (v[0] is key jb); works from registers, so the accumulator is not needed again
@@ -549,8 +635,21 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       //   lse2 = M + log2 Zt,   entropy = ln2 (log2 Zt - Xt / Zt)                (Eq. 4, one row)
       // lse_s holds -lse2; padded rows get -inf so that they contribute 2^(-inf) = 0.
       {
-        pdl_wait();
         const int ct = (int)threadIdx.x - 64;
+        if (p.fold) {
+          // operands of the extra K-step: zero both, then 1.0 in the first three K columns of the
+          // key-side operand (the row side is written after the merge below)
+          uint4* ext = reinterpret_cast<uint4*>(sm + L::kMergeOff + 4096);
+          for (int i = ct; i < (4096 + 8192) / 16; i += kComputeThreads) ext[i] = make_uint4(0u, 0u, 0u, 0u);
+          asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+          if (ct < kKeyTile) {
+            unsigned char* ax = sm + L::kMergeOff + 4096;
+#pragma unroll
+            for (int k = 0; k < 3; ++k)
+              *reinterpret_cast<__nv_bfloat16*>(ax + k16_offset(ct, k)) = __float2bfloat16_rn(1.0f);
+          }
+        }
+        pdl_wait();
         const int r = ct & (kRowBlock - 1), hp = ct >> 8;
         const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
         const int parts = p.segs;
@@ -602,8 +701,23 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
           }
           if (r < rows_here && seg == 0) p.row_ent[row] = ent;
           lse_s[r] = nlse;
+          if (p.fold) {
+            // -lse / c2 as hi + mid + lo (bf16 each: 24 bits together); padded rows get a huge
+            // negative value so that their 2^x is 0
+            const float Lv = nlse == -INFINITY ? -1.0e30f : nlse * p.inv_c2;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(Lv);
+            const float r1 = Lv - __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            unsigned char* bx = sm + L::kMergeOff + 8192;
+            *reinterpret_cast<__nv_bfloat16*>(bx + k16_offset(r, 0)) = hi;
+            *reinterpret_cast<__nv_bfloat16*>(bx + k16_offset(r, 1)) = mid;
+            *reinterpret_cast<__nv_bfloat16*>(bx + k16_offset(r, 2)) = lo;
+          }
         }
+        if (p.fold) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
         asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+        if (p.fold && ct == 0) mbar_arrive(bars + 8 * kBarExt);
       }
       // This thread owns key (tile * 128 + quarter * 32 + lane).  Rows: for W <= 64 the block's
       // rows [sub * 64, sub * 64 + 64) of every tile (two heads at W = 32, one at W = 64); for
@@ -617,7 +731,29 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       const int h0 = g * p.group + row0 / p.window;          // (first) head of this thread
       // sum over the chunk's 32 rows of 2^(x - lse) for this thread's key, all rows visible
       // (packed arithmetic; lse_s holds -lse)
+      auto pair_sum = [&](uint64_t s2, int pr, uint64_t x2) {
+        uint64_t p2;
+        if ((pr & 7) < kPoly2) {
+          float x0, x1;
+          unpack2(x2, x0, x1);
+          p2 = exp2_poly2(pack2(fminf(fmaxf(x0, -125.f), 126.f), fminf(fmaxf(x1, -125.f), 126.f)));
+        } else {
+          p2 = exp2_sfu2(x2);
+        }
+        return add2(s2, p2);
+      };
+      // the same sum when the MMA has already subtracted lse / c2: x = c2 * accumulator
+      auto colsum_folded = [&]() {
+        const uint64_t c22 = pack2(p.c2, p.c2), zero2 = pack2(0.f, 0.f);
+        uint64_t s2 = zero2;
+#pragma unroll
+        for (int pr = 0; pr < 16; ++pr) s2 = pair_sum(s2, pr, fma2(pack2(v[2 * pr], v[2 * pr + 1]), c22, zero2));
+        float a, b;
+        unpack2(s2, a, b);
+        return a + b;
+      };
       auto colsum = [&](int c) {
+        if (p.fold) return colsum_folded();
         const ulonglong2* l2 = reinterpret_cast<const ulonglong2*>(lse_s + col0 + c * 32);
         const uint64_t c22 = pack2(p.c2, p.c2);
         uint64_t s2 = pack2(0.f, 0.f);
@@ -627,16 +763,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
             const int pr = 2 * e4 + q;
-            const uint64_t x2 = fma2(pack2(v[2 * pr], v[2 * pr + 1]), c22, q == 0 ? l.x : l.y);
-            uint64_t p2;
-            if ((pr & 7) < kPoly2) {
-              float x0, x1;
-              unpack2(x2, x0, x1);
-              p2 = exp2_poly2(pack2(fminf(fmaxf(x0, -125.f), 126.f), fminf(fmaxf(x1, -125.f), 126.f)));
-            } else {
-              p2 = exp2_sfu2(x2);
-            }
-            s2 = add2(s2, p2);
+            s2 = pair_sum(s2, pr, fma2(pack2(v[2 * pr], v[2 * pr + 1]), c22, q == 0 ? l.x : l.y));
           }
         }
         float a, b;
@@ -649,7 +776,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const int i = (row0 + c * 32 + e) % p.window;
-          const float x = fmaf(v[e], p.c2, lse_s[col0 + c * 32 + e]);
+          const float x = fmaf(v[e], p.c2, p.fold ? 0.f : lse_s[col0 + c * 32 + e]);
           s += (i >= i_min) ? fast_exp2(x) : 0.f;
         }
         return s;
@@ -817,6 +944,9 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   if (segs > kMaxParts) segs = kMaxParts;           // pass 1 leaves one partial statistic per segment
   p.segs = segs;
   p.c2 = a.scale * kLog2e;
+  // the fold needs a finite lse / c2 (a zero scale keeps the plain form)
+  p.fold = (SKV_FOLD != 0) && pass == 2 && fabsf(p.c2) > 1e-20f ? 1 : 0;
+  p.inv_c2 = p.fold ? 1.0f / p.c2 : 0.f;
   p.row_part = ctx.ws.row_part;
   p.row_ent = ctx.ws.row_ent;
   p.cols = a.cols;

@@ -21,7 +21,7 @@ class Prefill:
                  seq: int, kv_budget: int, struct_budget: int, dtype: torch.dtype,
                  hidden_dim: int = 0, device: str = "cuda:0", lam: float = PAPER_LAMBDA,
                  weights: Sequence[float] = PAPER_WEIGHTS, l_limit: int = -1, flags: int = 0,
-                 keep_kv: bool = True):
+                 keep_kv: bool = True, defer_head_stats: bool = True):
         self.L, self.H, self.Hkv, self.d, self.w, self.N = n_layers, n_q_heads, n_kv_heads, head_dim, window, seq
         self.kv_budget, self.struct_budget = kv_budget, struct_budget
         self.lam, self.weights, self.l_limit, self.flags = lam, tuple(weights), l_limit, flags
@@ -47,19 +47,40 @@ class Prefill:
         self.pos_out = torch.empty((struct_budget,), dtype=i32, device=dev)
         self.pivot = -1
         self.transition: List[float] = []
+        # Eq. 5-6 of all layers in one batched call before the pivot (instead of a chain of short
+        # dependent launches after every layer): the pooled per-head attention of every layer is kept
+        self.defer = bool(defer_head_stats) and not (flags & binding.FLAG_NO_HEAD_STATS) and n_layers <= 128
+        self.head_cols = (torch.empty((n_layers, n_q_heads, seq), dtype=f32, device=dev) if self.defer else None)
+        self._stats_done = 0
 
     # -- Algorithm 1 lines 3-6 for one layer
     def score(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, scale: float,
               head_cols_out: Optional[torch.Tensor] = None) -> None:
         if layer == 0:
             self.c_running.zero_()
+            self._stats_done = 0
+        if self.defer:
+            self.ctx.score_layer(q_win, k, scale, self.s_hist[layer], self.metrics[layer],
+                                 c_inout=self.c_running, lam=self.lam, head_cols_out=self.head_cols[layer],
+                                 flags=self.flags | binding.FLAG_NO_HEAD_STATS)
+            if head_cols_out is not None:
+                head_cols_out.copy_(self.head_cols[layer])
+            return
         self.ctx.score_layer(q_win, k, scale, self.s_hist[layer], self.metrics[layer],
                              c_inout=self.c_running, lam=self.lam, head_cols_out=head_cols_out,
                              flags=self.flags)
 
+    def finish_scores(self, n_scored: Optional[int] = None) -> None:
+        """Sparsity and variance (Eq. 5-6) of the layers scored so far, in one batched call."""
+        L = self.L if n_scored is None else n_scored
+        if self.defer and self._stats_done < L:
+            self.ctx.head_stats(self.head_cols[self._stats_done:L], self.metrics[self._stats_done:L])
+            self._stats_done = L
+
     # -- Algorithm 1 lines 7-10 and 16: pivot, centrality at the pivot, both index sets
     def detect_and_select(self, n_scored: Optional[int] = None) -> int:
         L = self.L if n_scored is None else n_scored
+        self.finish_scores(L)
         self.pivot, self.transition = self.ctx.pivot(self.metrics[:L], self.weights, self.l_limit)
         self.ctx.accumulate(self.s_hist, self.pivot, self.lam, self.c_star)
         self.ctx.select(self.c_star, self.struct_budget, self.w, self.i_struct)

@@ -214,3 +214,24 @@ def test_hidden_state_gather_at_full_width(mods, cuda_device):
     assert np.array_equal(out.view(torch.int16).cpu().numpy(), O.compact(hid_bits, idx_np))
     assert np.array_equal(pout.cpu().numpy().ravel(), idx_np)
     ctx.close()
+
+
+def test_batched_head_statistics_equal_the_per_layer_ones(mods, cuda_device):
+    """Eq. 5-6 computed for all layers in one structkv_head_stats call (the pipeline's default)
+    give the very bits the per-layer computation inside structkv_score_layer gives."""
+    binding, pipeline = mods
+    wl = synth.WORKLOADS["llama32k"].scaled(5000 + 3, n_layers=5, n_hubs=8, budgets=(300,))
+    pl = synth.plan(wl)
+    layers = gpu_layers(wl, pl, cuda_device)
+    outs = []
+    for defer in (True, False):
+        pf = pipeline.Prefill(wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq,
+                              wl.budget, wl.struct_budget(), torch.bfloat16, device=cuda_device,
+                              defer_head_stats=defer)
+        assert pf.defer == defer
+        pf.run(layers)
+        torch.cuda.synchronize()
+        assert pf.ctx.poll_device_status() == binding.OK
+        outs.append((pf.metrics.clone(), pf.s_hist.clone(), pf.pivot))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and outs[0][2] == outs[1][2]
+    assert not torch.isnan(outs[0][0]).any()
