@@ -140,6 +140,7 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   a.q = q_window; a.k = k;
   a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
   a.n_keys = n_keys; a.scale = scale;
+  a.batch = 1; a.total_keys = n_keys; a.cu_seqlens = nullptr;
   a.cols = head_cols_out ? head_cols_out : c.ws.cols;
   a.col_stride = head_cols_out ? (long long)n_keys : (long long)c.n_pad;
 

@@ -12,6 +12,7 @@ namespace skv {
 constexpr int kKeyTile = 128;        // keys per tile in every scorer
 constexpr int kMaxParts = 160;       // upper bound on key segments per score row
 constexpr int kRowBlock = 256;       // score rows (head, window row) per tensor-core row block
+constexpr int kMaxBatch = 32;        // sequences one batched scoring call may hold
 constexpr int kMaxStatLayers = 128;  // layers one batched head-statistics call may cover
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -48,7 +49,10 @@ struct ScoreArgs {
   const void* q;            // [H, w, d]
   const void* k;
   long long k_stride_head, k_stride_token;   // elements
-  int n_keys;
+  int n_keys;               // keys of the sequence (a plain call), unused for a batch
+  int batch;                // sequences in the call (1 for a plain call)
+  int total_keys;           // rows of K along the token axis: n_keys, or cu_seqlens[batch]
+  const int* cu_seqlens;    // host, [batch + 1] first key of every sequence in the packed K; NULL = plain call
   float scale;
   float* cols;              // [H][col_stride] pooled per-head attention (output of pass 2)
   long long col_stride;

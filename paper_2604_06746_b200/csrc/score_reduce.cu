@@ -67,7 +67,8 @@ finalize_rows(const float4* __restrict__ row_part, int parts, int rows_pad, int 
 }
 
 // S_j = sum over heads (fixed order) of cols[h][j];  C_j <- lambda C_j + S_j  (Eq. 2, Eq. 3).
-// Four keys per thread where the layout allows 16-byte accesses.  Block 0 also finishes the
+// Four keys per thread where the layout allows 16-byte accesses.  NOTE: the order in which heads
+// are added differs between the two instantiations (grouped vs. sequential).  Block 0 also finishes the
 // layer's metrics: metrics[0] = mean entropy of the valid score rows (Eq. 4); metrics[1] = mean
 // over heads of the top-mass (Eq. 5), metrics[2] = mean over heads of (sum of squared deviations
 // from 1/n) / n (Eq. 6), both from head_part, or NaN when head statistics are not computed here.
@@ -82,24 +83,39 @@ reduce_finish(const float* __restrict__ cols, long long col_stride, int H, int n
   __shared__ float red[33];
   pdl_trigger();
   pdl_wait();
-  const int j = (blockIdx.x * kRcThreads + threadIdx.x) * VEC;
   if (VEC == 4) {
-    if (j < n) {                                   // n is a multiple of 4 in this instantiation
-      float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 8
-      for (int h = 0; h < H; ++h) {
-        const float4 v = *reinterpret_cast<const float4*>(cols + (size_t)h * col_stride + j);
+    // 64 threads along the keys (four keys each) x 4 groups of heads: four times the loads in
+    // flight; the groups' partial sums are added in group order (fixed order, deterministic)
+    __shared__ float4 part[3][64];
+    const int lane_j = threadIdx.x & 63, grp = threadIdx.x >> 6;
+    const int j4 = (blockIdx.x * 64 + lane_j) * 4;
+    const int h_per = (H + 3) / 4, h_lo = grp * h_per, h_hi = min(H, h_lo + h_per);
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j4 < n) {                                  // n is a multiple of 4 in this instantiation
+#pragma unroll 4
+      for (int h = h_lo; h < h_hi; ++h) {
+        const float4 v = *reinterpret_cast<const float4*>(cols + (size_t)h * col_stride + j4);
         s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
       }
-      *reinterpret_cast<float4*>(s_out + j) = s;
+    }
+    if (grp > 0) part[grp - 1][lane_j] = s;
+    __syncthreads();
+    if (grp == 0 && j4 < n) {
+#pragma unroll
+      for (int k = 0; k < 3; ++k) {
+        const float4 o = part[k][lane_j];
+        s.x += o.x; s.y += o.y; s.z += o.z; s.w += o.w;
+      }
+      *reinterpret_cast<float4*>(s_out + j4) = s;
       if (c_inout) {
-        float4 c = *reinterpret_cast<const float4*>(c_inout + j);
+        float4 c = *reinterpret_cast<const float4*>(c_inout + j4);
         c.x = fmaf(lambda, c.x, s.x); c.y = fmaf(lambda, c.y, s.y);
         c.z = fmaf(lambda, c.z, s.z); c.w = fmaf(lambda, c.w, s.w);
-        *reinterpret_cast<float4*>(c_inout + j) = c;
+        *reinterpret_cast<float4*>(c_inout + j4) = c;
       }
     }
-  } else if (j < n) {
+  } else if (blockIdx.x * kRcThreads + threadIdx.x < n) {
+    const int j = blockIdx.x * kRcThreads + threadIdx.x;
     float s = 0.f;
     for (int h = 0; h < H; ++h) s += cols[(size_t)h * col_stride + j];
     s_out[j] = s;
@@ -130,8 +146,8 @@ reduce_finish(const float* __restrict__ cols, long long col_stride, int H, int n
 // Per head: sum of squared deviations from 1/n (Eq. 6: the pooled vector sums to 1, so 1/n is its
 // mean; summing deviations instead of squares keeps near-uniform attention from cancelling) and
 // the mass of the k_rho largest entries (Eq. 5) of the pooled attention vector.  A cluster of
-// kHsCluster CTAs shares one head; each CTA owns a slice of the keys.  All entries are >= 0, so the unsigned order of the fp32 bit patterns is the
-// order of the values.  Two counting sweeps locate the k_rho-th largest value to 22 bits
+// CL CTAs shares one head; each CTA owns a slice of the keys.  All entries are >= 0, so the
+// unsigned order of the fp32 bit patterns is the order of the values.  Two counting sweeps locate the k_rho-th largest value to 22 bits
 // (histograms are merged in CTA 0 of the cluster through distributed shared memory with
 // integer atomics, so the result does not depend on arrival order):
 //   sweep 1: histogram of bits 30..20 (exponent + 3 mantissa bits); sum of squared deviations
@@ -139,14 +155,15 @@ reduce_finish(const float* __restrict__ cols, long long col_stride, int H, int n
 //            bits 19..9 of the entries inside it
 // The entries inside the threshold bin are then summed as count x bin midpoint: bins of the
 // second level are 2^-14 wide relative to their value, far inside the metric's tolerance.
-constexpr int kHsCluster = 8;
+constexpr int kHsCluster = 8;      // CTAs per (layer, head) when few vectors are in flight (one layer at a time)
 constexpr int kHsThreads = 1024;
 constexpr int kHsBins = 2048;
 constexpr int kHsCopies = 8;      // each bin is kept 8 times (lane & 7) so that a warp's hits on one bin spread
 constexpr int kHsItems = 16;      // entries per thread kept in registers between the sweeps
 
 // Shared memory of head_stats: hist[kHsBins][kHsCopies] | merged[2][kHsBins] (dynamic, 80 KB).
-__global__ void __cluster_dims__(kHsCluster, 1, 1) __launch_bounds__(kHsThreads)
+template <int CL>     // CTAs that share one (layer, head) vector: kHsCluster, or 1 when a batch of layers fills the GPU
+__global__ void __launch_bounds__(kHsThreads)
 head_stats(const float* __restrict__ cols, long long layer_stride, long long col_stride, int H, int n,
            int k_rho, float* __restrict__ head_part) {
   extern __shared__ unsigned hs_smem[];
@@ -158,10 +175,10 @@ head_stats(const float* __restrict__ cols, long long layer_stride, long long col
   __shared__ unsigned sel_bin, sel_rem;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
-  const int head = blockIdx.x / kHsCluster;          // (layer, head) pair: one cluster each
+  const int head = blockIdx.x / CL;                  // (layer, head) pair: one cluster each
   const float* a = cols + (size_t)(head / H) * layer_stride + (size_t)(head % H) * col_stride;
   const int tid = threadIdx.x, copy = tid & (kHsCopies - 1);
-  const int per = (n + kHsCluster - 1) / kHsCluster;
+  const int per = (n + CL - 1) / CL;
   const int lo = rank * per, hi = min(n, lo + per);
   const bool in_regs = per <= kHsItems * kHsThreads;  // otherwise the second sweep reads memory again
   unsigned* merged0 = cluster.map_shared_rank(merged, 0);
@@ -254,7 +271,7 @@ head_stats(const float* __restrict__ cols, long long layer_stride, long long col
     const float tot_in_bin = block_sum_1024(in_bin, red);
     if (tid == 0) {
       float s2 = 0.f, m = 0.f;
-      for (int r = 0; r < kHsCluster; ++r) { s2 += slots[2 * r]; m += slots[2 * r + 1]; }
+      for (int r = 0; r < CL; ++r) { s2 += slots[2 * r]; m += slots[2 * r + 1]; }
       head_part[head * 4 + 0] = s2;
       head_part[head * 4 + 1] = m + tot_in_bin;
     }
@@ -299,15 +316,39 @@ cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+template <int CL>
+static cudaError_t launch_head_stats_cl(const float* cols, long long layer_stride, long long col_stride,
+                                        int n_layers, int H, int n, int k_rho, float* head_part, cudaStream_t st) {
+  const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
+  cudaError_t e = cudaFuncSetAttribute(head_stats<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_layers * H * CL);
+  cfg.blockDim = dim3(kHsThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = CL;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, head_stats<CL>, cols, layer_stride, col_stride, H, n, k_rho, head_part);
+}
+
+// One layer at a time the vectors are few and the kernel is a chain of latencies: a cluster of
+// CTAs per vector shortens it.  A batch of layers brings enough vectors to fill the GPU with one
+// CTA each, which avoids the cluster barriers and remote merges altogether.
 static cudaError_t launch_head_stats(const float* cols, long long layer_stride, long long col_stride, int n_layers,
-                                     int H, int n, float* head_part, cudaStream_t st) {
+                                     int H, int n, float* head_part, int sm_count, cudaStream_t st) {
   int k_rho = n / 10;
   if (k_rho < 1) k_rho = 1;
-  const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
-  cudaError_t e = cudaFuncSetAttribute(head_stats, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(head_stats, dim3(n_layers * H * kHsCluster), dim3(kHsThreads), smem, st, cols, layer_stride,
-                    col_stride, H, n, k_rho, head_part);
+  if ((long long)n_layers * H >= 2ll * sm_count)
+    return launch_head_stats_cl<1>(cols, layer_stride, col_stride, n_layers, H, n, k_rho, head_part, st);
+  return launch_head_stats_cl<kHsCluster>(cols, layer_stride, col_stride, n_layers, H, n, k_rho, head_part, st);
 }
 
 cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long col_stride, int n, float lambda,
@@ -315,7 +356,7 @@ cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long co
                                  cudaStream_t st) {
   const int H = ctx.cfg.n_q_heads;
   if (with_head_stats) {
-    const cudaError_t e = launch_head_stats(cols, 0, col_stride, 1, H, n, ctx.ws.head_part, st);
+    const cudaError_t e = launch_head_stats(cols, 0, col_stride, 1, H, n, ctx.ws.head_part, ctx.sm_count, st);
     if (e != cudaSuccess) return e;
   }
   const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
@@ -323,7 +364,7 @@ cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long co
   const bool vec = n % 4 == 0 && col_stride % 4 == 0 && ((uintptr_t)cols % 16) == 0 &&
                    ((uintptr_t)s_out % 16) == 0 && ((uintptr_t)c_inout % 16) == 0;
   if (vec)
-    return launch_pdl(reduce_finish<4>, dim3((n / 4 + kRcThreads - 1) / kRcThreads), dim3(kRcThreads), 0, st, cols,
+    return launch_pdl(reduce_finish<4>, dim3((n / 4 + 63) / 64), dim3(kRcThreads), 0, st, cols,
                       col_stride, H, n, lambda, s_out, c_inout, (const float*)ctx.ws.row_ent, ctx.rows_pad,
                       rows_pg_pad, rows_pg, ctx.rows, (const float*)ctx.ws.head_part, with_head_stats ? 1 : 0,
                       metrics);
@@ -336,7 +377,7 @@ cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long co
 cudaError_t launch_head_stats_batch(const Ctx& ctx, const float* cols, long long layer_stride, long long col_stride,
                                     int n_layers, int n, float* metrics, cudaStream_t st) {
   const int H = ctx.cfg.n_q_heads;
-  cudaError_t e = launch_head_stats(cols, layer_stride, col_stride, n_layers, H, n, ctx.ws.head_part, st);
+  cudaError_t e = launch_head_stats(cols, layer_stride, col_stride, n_layers, H, n, ctx.ws.head_part, ctx.sm_count, st);
   if (e != cudaSuccess) return e;
   return launch_pdl(head_metrics, dim3((n_layers + 63) / 64), dim3(64), 0, st, (const float*)ctx.ws.head_part,
                     n_layers, H, n, metrics);

@@ -34,14 +34,22 @@ constexpr int kTcThreads = 64 + kComputeThreads;   // TMA warp, MMA warp, comput
 constexpr unsigned long long kWaitCycles = 1000000000ull;   // about 0.5 s at the maximum SM clock
 constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 0 * x stays finite
 
+// One sequence of a call: its keys are rows [key0, key0 + n_keys) of the packed K, its CTAs are
+// [cta0, cta0 + units * segs) of the grid.  A plain call is a batch of one.
+struct SeqDesc { int key0, n_keys, cta0, segs; };
+
 struct TcParams {
-  int n_keys, window, group, rows_pg, rows_pg_pad, rows_pad, n_rb, segs, n_tiles, n_pairs;
+  int window, group, rows_pg, rows_pg_pad, rows_pad, n_rb;
+  int n_seq;                           // sequences in this launch
+  int q_rows;                          // score rows of one sequence in the Q tensor (H * w)
+  long long rows_all;                  // n_seq * rows_pad: stride between segments in row_part
+  SeqDesc seq[kMaxBatch];
   float c2;                            // scale * log2(e)
   float inv_c2;                        // 1 / c2, or 0 when the fold of -lse into the MMA is off
   int fold;                            // pass 2: the accumulator already holds q.k - lse / c2
-  float4* row_part;                    // pass 1 out, pass 2 in: [segs][rows_pad] (ref, Z, U, -)
-  float* row_ent;                      // pass 2 out (segment 0 only): entropy of each score row, nats
-  float* cols;                         // pass 2 out [H][col_stride]
+  float4* row_part;                    // pass 1 out, pass 2 in: [segs][n_seq][rows_pad] (ref, Z, U, -)
+  float* row_ent;                      // pass 2 out (segment 0 only): [n_seq][rows_pad] entropy of each score row, nats
+  float* cols;                         // pass 2 out [H][col_stride], sequence b at column key0_b
   long long col_stride;
   int* status;
 };
@@ -238,14 +246,14 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
 // In pass 1, of every 8 consecutive elements (element pairs in the packed form) the first kPoly1
 // take the polynomial.
 #ifndef SKV_POLY1
-#define SKV_POLY1 0
+#define SKV_POLY1 1
 #endif
 #ifndef SKV_PACK1
-#define SKV_PACK1 0
+#define SKV_PACK1 1
 #endif
 // Pass 2: subtract lse inside the MMA (one extra K-step) instead of loading it from shared memory.
 #ifndef SKV_FOLD
-#define SKV_FOLD 0
+#define SKV_FOLD 1
 #endif
 constexpr int kPoly1 = SKV_POLY1;
 // In pass 2, of every 8 consecutive element pairs the first kPoly2 take the polynomial, the
@@ -314,7 +322,7 @@ enum { kBarFull = 0, kBarEmpty = kStages, kBarQ = 2 * kStages, kBarAccFull = 2 *
 template <int D, int PASS, int W>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-         const TcParams p) {
+         const __grid_constant__ TcParams p) {
   using L = Smem<D>;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -327,12 +335,18 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   volatile int* mma_in_flight = reinterpret_cast<volatile int*>(sm + L::kBarOff + 8 * kBarCount + 16);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int unit = blockIdx.x / p.segs, seg = blockIdx.x - unit * p.segs;
+  int sq = 0;                                                // the sequence this CTA works on
+  while (sq + 1 < p.n_seq && (int)blockIdx.x >= p.seq[sq + 1].cta0) ++sq;
+  const int n_keys = p.seq[sq].n_keys, key0 = p.seq[sq].key0, segs = p.seq[sq].segs;
+  const int cta = (int)blockIdx.x - p.seq[sq].cta0;
+  const int unit = cta / segs, seg = cta - unit * segs;
   const int g = unit / p.n_rb, rb = unit - g * p.n_rb;
+  const size_t row_base = (size_t)sq * p.rows_pad + (size_t)g * p.rows_pg_pad + rb * kRowBlock;
   // Pass 1 walks its segment in pairs of key tiles (256 keys per MMA), pass 2 in single tiles.
-  const int n_items = PASS == 1 ? p.n_pairs : p.n_tiles;
-  const int t_lo = (int)((long long)seg * n_items / p.segs);
-  const int t_hi = (int)((long long)(seg + 1) * n_items / p.segs);
+  const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
+  const int n_items = PASS == 1 ? (n_tiles + 1) / 2 : n_tiles;
+  const int t_lo = (int)((long long)seg * n_items / segs);
+  const int t_hi = (int)((long long)(seg + 1) * n_items / segs);
   const int n_my = t_hi - t_lo;
   // Pass 1 sweeps forward, pass 2 backward: the tiles pass 1 touched last are the ones still
   // in L2 when pass 2 starts.
@@ -373,7 +387,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     // ---------------- TMA producer ----------------
     if (lane == 0 && n_my > 0) {
       mbar_expect_tx(bars + 8 * kBarQ, L::kQBytes);
-      const int q_row0 = g * p.rows_pg + rb * kRowBlock;
+      const int q_row0 = sq * p.q_rows + g * p.rows_pg + rb * kRowBlock;
       for (int s = 0; s < L::kSub; ++s)
         tma_load_2d(base + L::kQOff + s * (L::kQBytes / L::kSub), &map_q, bars + 8 * kBarQ, s * 64, q_row0);
       int issued = 0;
@@ -383,12 +397,12 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         const uint32_t ph = (uint32_t)(t / kStages) & 1u;
         if (!mbar_wait_producer(bars + 8 * (kBarEmpty + s), ph ^ 1u, abort_flag, kWaitCycles)) break;
         mbar_expect_tx(bars + 8 * (kBarFull + s), L::kKBytes);
-        // a pair's second tile may lie wholly beyond the last key: TMA fills it with zeros and
-        // the causal mask discards it
+        // a tile may reach beyond the sequence's last key (into zero fill, or into the next
+        // sequence of a packed batch): the causal mask discards those keys
         const int tile = PASS == 1 ? 2 * t_lo + t : tile_of(t);
         for (int c = 0; c < L::kSub; ++c)
           tma_load_3d(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
-                      c * 64, tile * kKeyTile, g);
+                      c * 64, key0 + tile * kKeyTile, g);
         ++issued;
       }
       // drain: every copy this thread issued must have landed before the CTA may exit
@@ -470,7 +484,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     // a tile is "plain" when all of its keys are visible to every window row (j0 + 127 <= N - w);
     // the first (N - w + 1) / 128 tiles are
-    const int first_tail_tile = (p.n_keys - p.window + 1) / kKeyTile;
+    const int first_tail_tile = (n_keys - p.window + 1) / kKeyTile;
     float v[32];
     // lane 0 polls the barrier for its warp (bounded); the outcome is broadcast
     auto acc_full = [&](int t) {
@@ -497,8 +511,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       const uint64_t c22 = pack2(p.c2, p.c2);
       const int row_lo = quarter * 32 + lane;
       const int i_win = row_lo % p.window;          // window row of this thread's rows (the window divides 128)
-      const int t_pos = p.n_keys - p.window + i_win;                     // their position: they see keys <= t_pos
-      const int first_tail_pair = (p.n_keys - p.window + 1) / (2 * kKeyTile);
+      const int t_pos = n_keys - p.window + i_win;                     // their position: they see keys <= t_pos
+      const int first_tail_pair = (n_keys - p.window + 1) / (2 * kKeyTile);
       // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible;
       // of every 8 elements the first kPoly1 are exponentiated on the FMA pipe
       auto accumulate = [&](RowStat& r) {
@@ -622,7 +636,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
                 Z = fmaf(f, c[k].y, Z);
                 U = fmaf(f, fmaf(dm, c[k].y, c[k].z), U);
               }
-            p.row_part[(size_t)seg * p.rows_pad + g * p.rows_pg_pad + rb * kRowBlock + row_in_block] =
+            p.row_part[(size_t)seg * p.rows_all + row_base + row_in_block] =
                 make_float4(M, Z, U, 0.f);
           }
         }
@@ -651,8 +665,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         }
         pdl_wait();
         const int r = ct & (kRowBlock - 1), hp = ct >> 8;
-        const size_t row = (size_t)g * p.rows_pg_pad + rb * kRowBlock + r;
-        const int parts = p.segs;
+        const size_t row = row_base + r;
+        const int parts = segs;
         float M = -INFINITY, Zt = 0.f, Xt = 0.f;
         auto fold = [&](float ref_s, float Z_s, float X_s) {     // X_s = sum 2^(..)(.. - ref_s), relative to ref_s
           if (!(Z_s > 0.f)) return;
@@ -676,7 +690,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {
               const int sidx = s0 + 2 * b;
-              pv[b] = sidx < parts ? __ldg(&p.row_part[(size_t)sidx * p.rows_pad + row])
+              pv[b] = sidx < parts ? __ldg(&p.row_part[(size_t)sidx * p.rows_all + row])
                                    : make_float4(-INFINITY, 0.f, 0.f, 0.f);
             }
 #pragma unroll
@@ -786,7 +800,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         const int tile = tile_of(t);
         const int j = tile * kKeyTile + quarter * 32 + lane;
         const bool plain = tile < first_tail_tile;
-        const int i_min = j - (p.n_keys - p.window);        // window rows i < i_min do not see key j
+        const int i_min = j - (n_keys - p.window);        // window rows i < i_min do not see key j
         const uint32_t taddr = tmem + lane_base + (uint32_t)((t % kAccStages) * 256 + col0);
         const bool mine = warp_active && (W != 128 || (t & 1) == (sub >> 1));
         float sc[kChunks];
@@ -800,15 +814,15 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
           if (c == kChunks - 1) acc_release(t);             // every load of the tile has landed
           if (mine) sc[c] = plain ? colsum(c) : colsum_masked(c, i_min);
         }
-        if (mine && j < p.n_keys) {
+        if (mine && j < n_keys) {
           if (W == 32) {
-            p.cols[(size_t)h0 * p.col_stride + j] = sc[0] * inv_w;
-            if (row0 + 32 < p.rows_pg) p.cols[(size_t)(h0 + 1) * p.col_stride + j] = sc[1] * inv_w;
+            p.cols[(size_t)h0 * p.col_stride + key0 + j] = sc[0] * inv_w;
+            if (row0 + 32 < p.rows_pg) p.cols[(size_t)(h0 + 1) * p.col_stride + key0 + j] = sc[1] * inv_w;
           } else {
             float tot = 0.f;
 #pragma unroll
             for (int c = 0; c < kChunks; ++c) tot += sc[c];
-            p.cols[(size_t)h0 * p.col_stride + j] = tot * inv_w;
+            p.cols[(size_t)h0 * p.col_stride + key0 + j] = tot * inv_w;
           }
         }
       }
@@ -866,7 +880,7 @@ bool encode_maps(const Ctx& ctx, const ScoreArgs& a, CUtensorMap* mq, CUtensorMa
   TcState* s = (TcState*)ctx.tc;
   const int d = ctx.cfg.head_dim;
   {
-    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)ctx.cfg.n_q_heads * ctx.cfg.window};
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)a.batch * ctx.cfg.n_q_heads * ctx.cfg.window};
     cuuint64_t strides[1] = {(cuuint64_t)d * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)kRowBlock};
     cuuint32_t estr[2] = {1, 1};
@@ -876,11 +890,11 @@ bool encode_maps(const Ctx& ctx, const ScoreArgs& a, CUtensorMap* mq, CUtensorMa
       return false;
   }
   {
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)a.n_keys, (cuuint64_t)ctx.cfg.n_kv_heads};
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)a.total_keys, (cuuint64_t)ctx.cfg.n_kv_heads};
     cuuint64_t strides[2] = {(cuuint64_t)a.k_stride_token * 2, (cuuint64_t)a.k_stride_head * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)kKeyTile, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    if (ctx.cfg.n_kv_heads == 1) strides[1] = strides[0] * (cuuint64_t)a.n_keys;
+    if (ctx.cfg.n_kv_heads == 1) strides[1] = strides[0] * (cuuint64_t)a.total_keys;
     if (s->encode(mk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(a.k), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -928,21 +942,32 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   CUtensorMap mq, mk;
   if (!encode_maps(ctx, a, &mq, &mk)) return cudaErrorInvalidValue;
   TcParams p;
-  p.n_keys = a.n_keys;
   p.window = ctx.cfg.window;
   p.group = ctx.cfg.n_q_heads / ctx.cfg.n_kv_heads;
   p.rows_pg = p.group * p.window;
   p.rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
   p.rows_pad = ctx.rows_pad;
   p.n_rb = (p.rows_pg + kRowBlock - 1) / kRowBlock;
-  p.n_tiles = (a.n_keys + kKeyTile - 1) / kKeyTile;
+  p.n_seq = a.batch;
+  p.q_rows = ctx.cfg.n_q_heads * ctx.cfg.window;
+  p.rows_all = (long long)a.batch * ctx.rows_pad;
+  // The CTAs of the grid (about one per SM) are shared out over the sequences in proportion to
+  // their lengths; every (KV group, row block) unit of a sequence gets the same number of key
+  // segments, at least one, at most one per pair of key tiles.
   const int units = ctx.cfg.n_kv_heads * p.n_rb;
-  p.n_pairs = (p.n_tiles + 1) / 2;
-  int segs = ctx.sm_count / units;
-  if (segs < 1) segs = 1;
-  if (segs > p.n_pairs) segs = p.n_pairs;
-  if (segs > kMaxParts) segs = kMaxParts;           // pass 1 leaves one partial statistic per segment
-  p.segs = segs;
+  int grid = 0, max_segs = 0;
+  for (int b = 0; b < a.batch; ++b) {
+    const int key0 = a.cu_seqlens ? a.cu_seqlens[b] : 0;
+    const int n_b = a.cu_seqlens ? a.cu_seqlens[b + 1] - key0 : a.n_keys;
+    const int n_pairs = ((n_b + kKeyTile - 1) / kKeyTile + 1) / 2;
+    int segs = (int)((double)ctx.sm_count * n_b / ((double)a.total_keys * units));
+    if (segs < 1) segs = 1;
+    if (segs > n_pairs) segs = n_pairs;
+    if (segs > kMaxParts) segs = kMaxParts;         // pass 1 leaves one partial statistic per segment
+    p.seq[b] = SeqDesc{key0, n_b, grid, segs};
+    grid += units * segs;
+    if (segs > max_segs) max_segs = segs;
+  }
   p.c2 = a.scale * kLog2e;
   // the fold needs a finite lse / c2 (a zero scale keeps the plain form)
   p.fold = (SKV_FOLD != 0) && pass == 2 && fabsf(p.c2) > 1e-20f ? 1 : 0;
@@ -952,8 +977,7 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.cols = a.cols;
   p.col_stride = a.col_stride;
   p.status = ctx.ws.status;
-  *parts_out = segs;
-  const int grid = units * segs;
+  *parts_out = max_segs;
   const int d = ctx.cfg.head_dim, w = ctx.cfg.window;
   if (d == 128) return pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);
   return pass == 1 ? launch_w<64, 1>(w, mq, mk, p, grid, st) : launch_w<64, 2>(w, mq, mk, p, grid, st);
