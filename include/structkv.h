@@ -116,6 +116,52 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
                                      void* stream);
 
 /*
+ * One layer of observation-window scoring for a BATCH of prompts of different lengths
+ * (Section 4.1, implementation details: batches whose prompts reach their pivots at different
+ * layers are served with a padded addressing mask; every prompt is an independent problem with
+ * its own length, statistics, pivot and index sets).  The prompts' keys are packed back to back
+ * along the token axis; one launch per scorer pass covers all prompts, each prompt receiving a
+ * share of the grid in proportion to its length.  Per prompt the results equal those of
+ * structkv_score_layer on that prompt alone (same equations: Eq. 1, 2, 3, 4, 5, 6).
+ *
+ *   q_window      device, [batch, H, w, d] contiguous bf16.
+ *   k             device, packed keys: element (g, t, c) at k + g*k_stride_head + t*k_stride_token + c,
+ *                 prompt b owning tokens cu_seqlens[b] .. cu_seqlens[b+1]-1.
+ *   cu_seqlens    HOST, [batch + 1] ints, cu_seqlens[0] = 0, every length in [w, max_seq].
+ *   batch         1 .. 32.
+ *   s_out         device, [total] fp32 (total = cu_seqlens[batch]): S^(l) of every prompt, packed.
+ *   c_inout       device, [total] fp32 or NULL: C <- lambda*C + S, packed.
+ *   head_cols_out device, [H, total] fp32 or NULL.
+ *   metrics_out   device, [batch, 3] fp32: {entropy, sparsity, variance} of every prompt.
+ *   flags         STRUCTKV_FLAG_NO_HEAD_STATS or 0.
+ *   batch_workspace  device, 256-byte aligned, at least
+ *                 structkv_batch_workspace_bytes(cfg, batch, total) bytes, caller-owned; calls that
+ *                 share it must be ordered by the caller.
+ * Served by the tensor-core scorer only (bf16, window 32 / 64 / 128): other configurations
+ * return UNSUPPORTED.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.  Asynchronous on `stream`.
+ */
+size_t structkv_batch_workspace_bytes(const structkv_config* cfg, int max_batch, long long max_total_tokens);
+structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_window, const void* k,
+                                           long long k_stride_head, long long k_stride_token,
+                                           const int* cu_seqlens, int batch, float scale, float lambda,
+                                           float* s_out, float* c_inout, float* head_cols_out,
+                                           float* metrics_out, unsigned flags, void* batch_workspace,
+                                           size_t batch_workspace_bytes, void* stream);
+
+/*
+ * Eq. 10 / Eq. 13 for a batch of prompts of different lengths: prompt b selects budgets[b] tokens
+ * (window included) from its own scores scores[cu_seqlens[b] .. cu_seqlens[b+1]) and writes them,
+ * as positions inside that prompt, ascending, to idx_out + b*idx_stride; the remaining entries of
+ * the row are -1 (the padded addressing of a batch: padding is never a token).
+ *   cu_seqlens, budgets   HOST arrays, [batch + 1] and [batch]; window <= budgets[b] <= length of b.
+ *   idx_out               device, [batch, idx_stride] int32, idx_stride >= max budget.
+ * Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_select_batch(structkv_ctx* ctx, const float* scores, const int* cu_seqlens,
+                                      const int* budgets, int batch, int window, int* idx_out,
+                                      long long idx_stride, void* stream);
+
+/*
  * Eq. 5 and Eq. 6 (Section 3.3) for several layers at once, from the pooled per-head attention
  * that structkv_score_layer wrote to head_cols_out.  A caller that scores many layers passes
  * STRUCTKV_FLAG_NO_HEAD_STATS and a distinct head_cols_out slab per layer, then makes ONE call

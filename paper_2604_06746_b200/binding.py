@@ -52,6 +52,13 @@ lib.structkv_score_layer_static.restype = _i
 lib.structkv_score_layer_static.argtypes = [ctypes.POINTER(Config), _vp, _vp, _ll, _ll, _i, _f, _f, _vp, _vp,
                                             _vp, _vp, _u, _vp]
 STATIC_SCRATCH_BYTES = 8 << 20
+lib.structkv_batch_workspace_bytes.restype = ctypes.c_size_t
+lib.structkv_batch_workspace_bytes.argtypes = [ctypes.POINTER(Config), _i, _ll]
+lib.structkv_score_layer_batch.restype = _i
+lib.structkv_score_layer_batch.argtypes = [_vp, _vp, _vp, _ll, _ll, ctypes.POINTER(_i), _i, _f, _f, _vp, _vp, _vp,
+                                           _vp, _u, _vp, ctypes.c_size_t, _vp]
+lib.structkv_select_batch.restype = _i
+lib.structkv_select_batch.argtypes = [_vp, _vp, ctypes.POINTER(_i), ctypes.POINTER(_i), _i, _i, _vp, _ll, _vp]
 lib.structkv_head_stats.restype = _i
 lib.structkv_head_stats.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _vp, _vp]
 lib.structkv_pivot.restype = _i
@@ -170,6 +177,40 @@ class Context:
                                         k.shape[1], scale, lam, s_out.data_ptr(), _ptr(c_inout),
                                         _ptr(head_cols_out), metrics_out.data_ptr(), flags,
                                         _stream(stream)), "structkv_score_layer")
+
+    def score_layer_batch(self, q_window: torch.Tensor, k: torch.Tensor, cu_seqlens: Sequence[int], scale: float,
+                          s_out: torch.Tensor, metrics_out: torch.Tensor, workspace: torch.Tensor,
+                          c_inout: Optional[torch.Tensor] = None, lam: float = 0.9,
+                          head_cols_out: Optional[torch.Tensor] = None, flags: int = 0,
+                          stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_score_layer_batch: ``q_window [B, H, w, d]``, ``k [H_kv, total, d]`` packed prompts,
+        ``cu_seqlens`` host ints ``[B + 1]``."""
+        B = len(cu_seqlens) - 1
+        assert q_window.is_contiguous() and q_window.shape[0] == B and k.stride(2) == 1
+        assert k.shape[1] == cu_seqlens[-1] and s_out.numel() == cu_seqlens[-1] and metrics_out.shape == (B, 3)
+        cu = (_i * (B + 1))(*cu_seqlens)
+        _check(lib.structkv_score_layer_batch(self._h, q_window.data_ptr(), k.data_ptr(), k.stride(0), k.stride(1),
+                                              cu, B, scale, lam, s_out.data_ptr(), _ptr(c_inout),
+                                              _ptr(head_cols_out), metrics_out.data_ptr(), flags,
+                                              workspace.data_ptr(), workspace.numel(), _stream(stream)),
+               "structkv_score_layer_batch")
+
+    def batch_workspace(self, max_batch: int, max_total_tokens: int) -> torch.Tensor:
+        n = lib.structkv_batch_workspace_bytes(ctypes.byref(self.cfg), max_batch, max_total_tokens)
+        if n == 0:
+            raise StructKVError(ERR_INVALID_ARG, "structkv_batch_workspace_bytes")
+        return torch.empty(n, dtype=torch.uint8, device=self.device)
+
+    def select_batch(self, scores: torch.Tensor, cu_seqlens: Sequence[int], budgets: Sequence[int], window: int,
+                     idx_out: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_select_batch: packed ``scores [total]`` -> ``idx_out [B, stride]`` int32, padded with -1."""
+        B = len(budgets)
+        assert scores.is_contiguous() and scores.dtype == torch.float32
+        assert idx_out.dtype == torch.int32 and idx_out.is_contiguous() and idx_out.shape[0] == B
+        cu = (_i * (B + 1))(*cu_seqlens)
+        bu = (_i * B)(*budgets)
+        _check(lib.structkv_select_batch(self._h, scores.data_ptr(), cu, bu, B, window, idx_out.data_ptr(),
+                                         idx_out.stride(0), _stream(stream)), "structkv_select_batch")
 
     def head_stats(self, head_cols: torch.Tensor, metrics: torch.Tensor,
                    stream: Optional[torch.cuda.Stream] = None) -> None:

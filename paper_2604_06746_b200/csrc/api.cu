@@ -161,6 +161,117 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   return e == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
 }
 
+// ---- batches of prompts of different lengths (packed along the token axis) ------------------
+namespace skv {
+struct BatchWs { float4* row_part; float* row_ent; float* cols; float* head_part; size_t bytes; };
+static BatchWs carve_batch(const structkv_config& cfg, int max_batch, long long max_total, void* base) {
+  BatchWs w{};
+  char* p = (char*)base;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* r = p ? (void*)(p + off) : nullptr;
+    off += align_up(bytes, 256);
+    return r;
+  };
+  const size_t rows_all = (size_t)max_batch * rows_pad_of(cfg);
+  const size_t t_pad = align_up((size_t)max_total, kKeyTile);
+  w.row_part = (float4*)take((size_t)kMaxParts * rows_all * sizeof(float4));
+  w.row_ent = (float*)take(rows_all * sizeof(float));
+  w.cols = (float*)take((size_t)cfg.n_q_heads * t_pad * sizeof(float));
+  w.head_part = (float*)take((size_t)max_batch * cfg.n_q_heads * 4 * sizeof(float));
+  w.bytes = off;
+  return w;
+}
+}  // namespace skv
+
+size_t structkv_batch_workspace_bytes(const structkv_config* cfg, int max_batch, long long max_total_tokens) {
+  if (!cfg || !config_ok(*cfg) || !config_supported(*cfg)) return 0;
+  if (max_batch < 1 || max_batch > kMaxBatch || max_total_tokens < cfg->window || max_total_tokens > 0x7fffff00ll)
+    return 0;
+  return carve_batch(*cfg, max_batch, max_total_tokens, nullptr).bytes;
+}
+
+structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_window, const void* k,
+                                           long long k_stride_head, long long k_stride_token,
+                                           const int* cu_seqlens, int batch, float scale, float lambda,
+                                           float* s_out, float* c_inout, float* head_cols_out,
+                                           float* metrics_out, unsigned flags, void* batch_workspace,
+                                           size_t batch_workspace_bytes, void* stream) {
+  if (!ctx || !q_window || !k || !cu_seqlens || !s_out || !metrics_out) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch < 1 || batch > kMaxBatch) return STRUCTKV_ERR_INVALID_ARG;
+  Ctx& c = ctx->c;
+  const structkv_config& cfg = c.cfg;
+  if (cu_seqlens[0] != 0) return STRUCTKV_ERR_INVALID_ARG;
+  for (int b = 0; b < batch; ++b) {
+    const long long n_b = (long long)cu_seqlens[b + 1] - cu_seqlens[b];
+    if (n_b < cfg.window || n_b > cfg.max_seq) return STRUCTKV_ERR_INVALID_ARG;
+  }
+  const int total = cu_seqlens[batch];
+  if (!std::isfinite(scale) || !std::isfinite(lambda)) return STRUCTKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q_window % 16) || ((uintptr_t)k % 16)) return STRUCTKV_ERR_INVALID_ARG;
+  if (k_stride_token < cfg.head_dim || k_stride_head < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if ((k_stride_token * 2) % 16 || (k_stride_head * 2) % 16) return STRUCTKV_ERR_INVALID_ARG;
+  if (flags & ~STRUCTKV_FLAG_NO_HEAD_STATS) return STRUCTKV_ERR_INVALID_ARG;
+  const size_t need = carve_batch(cfg, batch, total, nullptr).bytes;
+  if (!batch_workspace || batch_workspace_bytes < need || ((uintptr_t)batch_workspace % 256) != 0)
+    return STRUCTKV_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const BatchWs bw = carve_batch(cfg, batch, total, batch_workspace);
+
+  Ctx view = c;                       // same device, tensor-map encoder and status word; batch-sized scratch
+  view.ws.row_part = bw.row_part;
+  view.ws.row_ent = bw.row_ent;
+  view.ws.cols = bw.cols;
+  view.ws.head_part = bw.head_part;
+  ScoreArgs a;
+  a.q = q_window; a.k = k;
+  a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
+  a.n_keys = 0; a.batch = batch; a.total_keys = total; a.cu_seqlens = cu_seqlens;
+  a.scale = scale;
+  a.cols = head_cols_out ? head_cols_out : bw.cols;
+  a.col_stride = head_cols_out ? (long long)total : (long long)align_up((size_t)total, kKeyTile);
+  // only the tensor-core scorer handles packed batches
+  if (cfg.dtype != STRUCTKV_BF16 || !tc_supported(view, a)) return STRUCTKV_ERR_UNSUPPORTED;
+  int parts = 0;
+  if (launch_score_tc(view, a, &parts, 1, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  if (launch_score_tc(view, a, &parts, 2, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  // per sequence: S = sum over heads, C <- lambda C + S, and the sequence's metric triple
+  for (int b = 0; b < batch; ++b) {
+    const int key0 = cu_seqlens[b], n_b = cu_seqlens[b + 1] - key0;
+    Ctx one = view;
+    one.ws.row_ent = bw.row_ent + (size_t)b * c.rows_pad;
+    one.ws.head_part = bw.head_part + (size_t)b * cfg.n_q_heads * 4;
+    if (launch_reduce_finish(one, a.cols + key0, a.col_stride, n_b, lambda, s_out + key0,
+                             c_inout ? c_inout + key0 : nullptr, !(flags & STRUCTKV_FLAG_NO_HEAD_STATS),
+                             metrics_out + 3 * b, st) != cudaSuccess)
+      return STRUCTKV_ERR_CUDA;
+  }
+  return STRUCTKV_OK;
+}
+
+structkv_status structkv_select_batch(structkv_ctx* ctx, const float* scores, const int* cu_seqlens,
+                                      const int* budgets, int batch, int window, int* idx_out,
+                                      long long idx_stride, void* stream) {
+  if (!ctx || !scores || !cu_seqlens || !budgets || !idx_out) return STRUCTKV_ERR_INVALID_ARG;
+  if (batch < 1 || batch > kMaxBatch || window < 0) return STRUCTKV_ERR_INVALID_ARG;
+  for (int b = 0; b < batch; ++b) {
+    const long long n_b = (long long)cu_seqlens[b + 1] - cu_seqlens[b];
+    if (n_b < 1 || budgets[b] < window || budgets[b] > n_b || budgets[b] > idx_stride)
+      return STRUCTKV_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  // padding entries read -1: no prompt ever addresses a batch-mate's tokens
+  if (cudaMemsetAsync(idx_out, 0xff, (size_t)batch * idx_stride * sizeof(int), st) != cudaSuccess)
+    return STRUCTKV_ERR_CUDA;
+  for (int b = 0; b < batch; ++b) {
+    const int key0 = cu_seqlens[b], n_b = cu_seqlens[b + 1] - key0;
+    if (launch_select(scores + key0, 0, 1, n_b, budgets[b], window, idx_out + (size_t)b * idx_stride, st) !=
+        cudaSuccess)
+      return STRUCTKV_ERR_CUDA;
+  }
+  return STRUCTKV_OK;
+}
+
 structkv_status structkv_head_stats(structkv_ctx* ctx, const float* head_cols, long long layer_stride,
                                     long long col_stride, int n_layers, int n, float* metrics,
                                     void* stream) {
