@@ -192,8 +192,7 @@ class Resident:
         if timed: e[1].record()
         pf.detect_and_select(len(layers))
         if timed: e[2].record()
-        for l, t in enumerate(layers):
-            pf.compact_kv(l, t["k"], t["v"], t.get("kv"))
+        pf.compact_all_kv(layers)
         pf.compact_hidden(self.hidden, self.positions)
         if timed: e[3].record()
         return e
@@ -330,10 +329,10 @@ def launches_per_step(wl, flags):
     from paper_2604_06746_b200 import binding
     # per layer: scorer pass 1, pass 2, column reduce + metrics (the CUDA-core scorer adds a row
     # finalisation); per step: batched head statistics (2), accumulate, 2 selections, one K/V gather
-    # per layer, hidden states, positions
+    # over all layers, hidden states, positions
     per_layer = 3 if wl.dtype == "bf16" else 4
     stats = 0 if (flags & binding.FLAG_NO_HEAD_STATS) else 2
-    return wl.n_layers * per_layer + stats + 1 + 2 + wl.n_layers + 2
+    return wl.n_layers * per_layer + stats + 1 + 2 + 1 + 2
 
 
 # ------------------------------------------------------------------------------------------------
@@ -476,8 +475,7 @@ def measure_e2e(res, dev, steps, world):
             main.wait_event(arrived[l])
             pf.score(l, t["q_win"], t["k"], t["scale"])
         pf.detect_and_select(len(layers))
-        for l, t in enumerate(layers):
-            pf.compact_kv(l, t["k"], t["v"], t.get("kv"))
+        pf.compact_all_kv(layers)
         main.wait_event(arrived[len(layers)])
         pf.compact_hidden(hidden, positions)
         done = torch.cuda.Event()

@@ -288,6 +288,22 @@ structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long s
                                  void* stream);
 
 /*
+ * structkv_compact (Algorithm 1 line 17) for several layers in ONE launch: layer l gathers rows of
+ * its own source srcs[l] at its own index list idx + l*idx_layer_stride into
+ * dst + l*dst_layer_stride_bytes, laid out [n_slabs, n_idx, row_bytes].  With small budgets a
+ * gather per layer is a chain of launches of a few microseconds each; one launch removes it.
+ *   srcs      HOST array of n_layers device pointers (1 .. 128 layers), all sources sharing
+ *             slab_stride_bytes, row_stride_bytes, row_bytes, n_slabs and n_rows_src.
+ *   idx       device, int32, n_idx entries per layer, idx_layer_stride >= n_idx.
+ * An out-of-range index copies nothing and records STRUCTKV_ERR_INVALID_ARG in the device status
+ * word.  Bit exact.  Errors: INVALID_ARG, CUDA.  Asynchronous on `stream`.
+ */
+structkv_status structkv_compact_layers(structkv_ctx* ctx, const void* const* srcs, int n_layers,
+                                        long long slab_stride_bytes, long long row_stride_bytes, int row_bytes,
+                                        int n_slabs, int n_rows_src, const int* idx, long long idx_layer_stride,
+                                        int n_idx, void* dst, long long dst_layer_stride_bytes, void* stream);
+
+/*
  * Per-KV-group saliency and per-slab gathers: the per-head variant of the cache selection.
  * Paper: Section 3.2, the sentence before Eq. 2 (attention is aggregated over the query heads
  * that share a KV head); Eq. 13 applied per KV head instead of per layer; and Section 4.1, the

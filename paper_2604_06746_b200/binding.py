@@ -72,6 +72,8 @@ lib.structkv_compact.restype = _i
 lib.structkv_compact.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _i, _vp, _i, _vp, _vp]
 lib.structkv_group_saliency.restype = _i
 lib.structkv_group_saliency.argtypes = [_vp, _vp, _ll, _i, _vp, _vp]
+lib.structkv_compact_layers.restype = _i
+lib.structkv_compact_layers.argtypes = [_vp, ctypes.POINTER(_vp), _i, _ll, _ll, _i, _i, _i, _vp, _ll, _i, _vp, _ll, _vp]
 lib.structkv_compact_per_slab.restype = _i
 lib.structkv_compact_per_slab.argtypes = [_vp, _vp, _ll, _ll, _i, _i, _i, _vp, _ll, _i, _vp, _vp]
 lib.structkv_block_scores.restype = _i
@@ -260,6 +262,25 @@ class Context:
         _check(lib.structkv_compact(self._h, src.data_ptr(), src.stride(0) * es, src.stride(1) * es,
                                     row_elems * es, src.shape[0], src.shape[1], idx.data_ptr(),
                                     idx.numel(), dst.data_ptr(), _stream(stream)), "structkv_compact")
+
+    def compact_layers(self, srcs: Sequence[torch.Tensor], idx: torch.Tensor, dst: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_compact_layers: every ``srcs[l] [n_slabs, n_rows, row...]`` (same shape and strides)
+        gathered at ``idx[l]`` into ``dst[l] [n_slabs, n_idx, row...]`` by one launch."""
+        L = len(srcs)
+        s0 = srcs[0]
+        assert idx.dtype == torch.int32 and idx.dim() == 2 and idx.shape[0] == L and idx.stride(1) == 1
+        assert dst.shape[0] == L and dst[0].is_contiguous()
+        assert all(t.shape == s0.shape and t.stride() == s0.stride() and t.dtype == s0.dtype for t in srcs)
+        row_elems = 1
+        for sdim in s0.shape[2:]:
+            row_elems *= sdim
+        es = s0.element_size()
+        ptrs = (_vp * L)(*[t.data_ptr() for t in srcs])
+        _check(lib.structkv_compact_layers(self._h, ptrs, L, s0.stride(0) * es, s0.stride(1) * es, row_elems * es,
+                                           s0.shape[0], s0.shape[1], idx.data_ptr(), idx.stride(0), idx.shape[1],
+                                           dst.data_ptr(), dst.stride(0) * es, _stream(stream)),
+               "structkv_compact_layers")
 
     def group_saliency(self, head_cols: torch.Tensor, out: torch.Tensor,
                        stream: Optional[torch.cuda.Stream] = None) -> None:

@@ -359,6 +359,23 @@ structkv_status structkv_compact(structkv_ctx* ctx, const void* src, long long s
              : STRUCTKV_ERR_CUDA;
 }
 
+structkv_status structkv_compact_layers(structkv_ctx* ctx, const void* const* srcs, int n_layers,
+                                        long long slab_stride_bytes, long long row_stride_bytes, int row_bytes,
+                                        int n_slabs, int n_rows_src, const int* idx, long long idx_layer_stride,
+                                        int n_idx, void* dst, long long dst_layer_stride_bytes, void* stream) {
+  if (!ctx || !srcs || !dst || !idx) return STRUCTKV_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > kMaxGatherLayers) return STRUCTKV_ERR_INVALID_ARG;
+  if (row_bytes < 1 || n_slabs < 0 || n_rows_src < 1 || n_idx < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if (row_stride_bytes < row_bytes || slab_stride_bytes < 0 || idx_layer_stride < n_idx) return STRUCTKV_ERR_INVALID_ARG;
+  if (dst_layer_stride_bytes < (long long)n_slabs * n_idx * row_bytes) return STRUCTKV_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!srcs[l]) return STRUCTKV_ERR_INVALID_ARG;
+  const Ctx& c = ctx->c;
+  return launch_compact_layers(srcs, n_layers, slab_stride_bytes, row_stride_bytes, row_bytes, n_slabs, n_rows_src,
+                               idx, idx_layer_stride, n_idx, dst, dst_layer_stride_bytes, c.ws.status, c.sm_count,
+                               (cudaStream_t)stream) == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
+}
+
 structkv_status structkv_compact_per_slab(structkv_ctx* ctx, const void* src, long long slab_stride_bytes,
                                           long long row_stride_bytes, int row_bytes, int n_slabs,
                                           int n_rows_src, const int* idx, long long idx_slab_stride,

@@ -13,7 +13,8 @@ constexpr int kKeyTile = 128;        // keys per tile in every scorer
 constexpr int kMaxParts = 160;       // upper bound on key segments per score row
 constexpr int kRowBlock = 256;       // score rows (head, window row) per tensor-core row block
 constexpr int kMaxBatch = 32;        // sequences one batched scoring call may hold
-constexpr int kMaxStatLayers = 128;  // layers one batched head-statistics call may cover
+constexpr int kMaxStatLayers = 128;
+constexpr int kMaxGatherLayers = 128; // layers one multi-layer gather may cover (their pointers are a kernel argument)  // layers one batched head-statistics call may cover
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -102,6 +103,10 @@ cudaError_t launch_compact(const void* src, long long slab_stride, long long row
                            int row_bytes, int n_slabs, int n_rows_src, const int* idx,
                            long long idx_slab_stride, int n_idx, void* dst, int* status, int sm_count,
                            cudaStream_t st);
+cudaError_t launch_compact_layers(const void* const* srcs, int n_layers, long long slab_stride, long long row_stride,
+                                  int row_bytes, int n_slabs, int n_rows_src, const int* idx,
+                                  long long idx_layer_stride, int n_idx, void* dst, long long dst_layer_stride,
+                                  int* status, int sm_count, cudaStream_t st);
 cudaError_t launch_group_saliency(const float* head_cols, long long col_stride, int n_heads, int group, int n,
                                   float* out, cudaStream_t st);
 

@@ -255,6 +255,10 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
 #ifndef SKV_FOLD
 #define SKV_FOLD 1
 #endif
+// Start-up offset between the compute warps of one scheduler (nanoseconds per column group).
+#ifndef SKV_STAGGER_NS
+#define SKV_STAGGER_NS 0
+#endif
 constexpr int kPoly1 = SKV_POLY1;
 // In pass 2, of every 8 consecutive element pairs the first kPoly2 take the polynomial, the
 // rest the special-function unit: the two pipes work side by side (2 of 8 measured best).
@@ -502,6 +506,11 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       if (lane == 0) mbar_arrive(bars + 8 * (kBarAccEmpty + t % kAccStages));
     };
 
+    // The four compute warps of a scheduler share a lane quarter and are released by the same
+    // barrier, so without help they load, compute and load again in step, and the exponential unit
+    // idles whenever all of them wait for tensor memory.  A start-up offset per column group
+    // spreads their phases; in steady state nothing brings them back in step.
+    if (SKV_STAGGER_NS > 0 && sub > 0) __nanosleep((unsigned)(sub * SKV_STAGGER_NS));
     if (PASS == 1) {
       // A unit's accumulator holds one 128-row half of the block x the pair's 256 keys.  This
       // thread owns row (quarter * 32 + lane) of BOTH halves (units alternate between them) and

@@ -99,6 +99,18 @@ class Prefill:
         self.ctx.compact(k, self.i_kv[layer], self.k_out[slot])
         self.ctx.compact(v, self.i_kv[layer], self.v_out[slot])
 
+    def compact_all_kv(self, layers: Sequence[Dict[str, torch.Tensor]]) -> None:
+        """Algorithm 1 line 17 for resident layers: one launch for all of them when every layer keeps
+        K and V in one joint allocation, else one gather per layer."""
+        if self.keep_kv and len(layers) <= 128 and all("kv" in t for t in layers):
+            self.ctx.compact_layers([t["kv"].view(2 * self.Hkv, t["kv"].shape[2], self.d) for t in layers],
+                                    self.i_kv[:len(layers)],
+                                    self.kv_out[:len(layers)].view(len(layers), 2 * self.Hkv, self.kv_budget, self.d))
+            return
+        for l, t in enumerate(layers):
+            if "v" in t:
+                self.compact_kv(l, t["k"], t["v"], t.get("kv"))
+
     # -- Algorithm 1 line 13
     def compact_hidden(self, hidden: torch.Tensor, positions: torch.Tensor) -> None:
         self.ctx.compact(hidden[None], self.i_struct, self.hidden_out[None])
@@ -140,9 +152,7 @@ class Prefill:
         for l, t in enumerate(layers):
             self.score(l, t["q_win"], t["k"], t["scale"])
         self.detect_and_select(len(layers))
-        for l, t in enumerate(layers):
-            if "v" in t:
-                self.compact_kv(l, t["k"], t["v"], t.get("kv"))
+        self.compact_all_kv(layers)
         if hidden is not None:
             self.compact_hidden(hidden, positions)
         return self.pivot

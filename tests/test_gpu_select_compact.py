@@ -130,3 +130,27 @@ def test_bounded_wait_expiry_is_reported_once(cuda_device):
     assert ctx.poll_device_status() == binding.OK
     assert idx[-1].item() == 4095
     ctx.close()
+
+
+def test_multi_layer_gather_equals_the_oracle_per_layer(ctx):
+    """structkv_compact_layers: several layers, each with its own source and index list, one launch."""
+    rng = np.random.default_rng(11)
+    L, slabs, n, d, b = 5, 6, 3000, 128, 257
+    srcs = [torch.from_numpy(rng.integers(-2 ** 15, 2 ** 15, size=(slabs, n, d), dtype=np.int16)).cuda() for _ in range(L)]
+    idx_np = np.stack([np.sort(rng.choice(n, size=b, replace=False)) for _ in range(L)]).astype(np.int32)
+    idx = torch.from_numpy(idx_np).cuda()
+    out = torch.zeros((L, slabs, b, d), dtype=torch.int16, device="cuda")
+    ctx.compact_layers(srcs, idx, out)
+    torch.cuda.synchronize()
+    from paper_2604_06746_b200 import binding
+    assert ctx.poll_device_status() == binding.OK
+    for l in range(L):
+        assert np.array_equal(out[l].cpu().numpy(), O.compact(srcs[l].cpu().numpy(), idx_np[l])), l
+    # odd row size (4-byte units) and a strided source
+    srcs2 = [torch.from_numpy(rng.integers(0, 255, size=(2, 500, 20), dtype=np.uint8)).cuda()[:, :, :12] for _ in range(3)]
+    idx2 = torch.from_numpy(np.stack([rng.permutation(500)[:40] for _ in range(3)]).astype(np.int32)).cuda()
+    out2 = torch.zeros((3, 2, 40, 12), dtype=torch.uint8, device="cuda")
+    ctx.compact_layers(srcs2, idx2, out2)
+    torch.cuda.synchronize()
+    for l in range(3):
+        assert np.array_equal(out2[l].cpu().numpy(), O.compact(srcs2[l].cpu().numpy(), idx2[l].cpu().numpy())), l

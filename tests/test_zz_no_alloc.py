@@ -53,6 +53,33 @@ def test_static_scratch_scoring_matches_context_scoring_twice(cuda_device, name,
     ctx.close()
 
 
+def test_static_scratch_scoring_allocates_nothing_and_serves_the_pooled_columns_itself(cuda_device):
+    """What the entry point exists for: after its first call on the device (which does the one-time
+    set-up) further calls leave the amount of free device memory untouched.  Also the variant
+    without head_cols_out, whose pooled per-head columns then live inside the fixed scratch."""
+    from paper_2604_06746_b200 import binding
+    wl = synth.WORKLOADS["llama32k"].scaled(4096 + 77, n_layers=1, n_hubs=8)
+    t = synth.make_layer(wl, synth.plan(wl), 0, device="cpu", with_v=False)
+    q, k = t["q_win"].to(cuda_device), t["k"].to(cuda_device)
+    f32 = torch.float32
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, torch.bfloat16, cuda_device)
+    s_ref, m_ref = torch.zeros(wl.seq, dtype=f32, device=cuda_device), torch.zeros(3, dtype=f32, device=cuda_device)
+    s_new, m_new = torch.zeros_like(s_ref), torch.zeros_like(m_ref)
+    ctx.score_layer(q, k, t["scale"], s_ref, m_ref)
+    args = (wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, q, k, t["scale"], s_new, m_new)
+    binding.score_layer_static(*args)                      # first call: one-time set-up happens here
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for _ in range(5):
+        binding.score_layer_static(*args)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    P.assert_scores_close(s_new.cpu().numpy(), s_ref.cpu().numpy(), "S without head_cols_out")
+    for c in range(3):
+        P.assert_metric_close(m_new[c].item(), m_ref[c].item(), f"metric {c} without head_cols_out")
+    ctx.close()
+
+
 def test_static_scratch_scoring_refuses_configurations_beyond_its_scratch(cuda_device):
     from paper_2604_06746_b200 import binding
     big = binding.Config(32, 8, 128, 64, 131072, binding.BF16)
