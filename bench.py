@@ -39,7 +39,7 @@ SFU_EXP_PER_CLK_PER_SM = 16      # special-function results per clock per SM (cc
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the scorer launches of one layer,
 # from an ncu capture of the current kernels; None = no capture of the current kernels exists.
 NCU_TRAFFIC_BYTES_PER_LAYER = None
-NCU_TRAFFIC_NOTE = "no ncu capture of the current scorer kernels yet"
+NCU_TRAFFIC_NOTE = "pending: single-pass ncu capture (caches left as the previous kernel leaves them) of the current kernels"
 
 
 def load_peaks():

@@ -140,6 +140,24 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// The same copy with an L2 eviction-priority hint for the lines it brings in.
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                                 int c1, int c2, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1) {
   asm volatile(
@@ -254,6 +272,10 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
 // Pass 2: subtract lse inside the MMA (one extra K-step) instead of loading it from shared memory.
 #ifndef SKV_FOLD
 #define SKV_FOLD 1
+#endif
+// Percentage of a pass-1 segment (its end) that L2 is asked to keep for pass 2; 0 = no hints.
+#ifndef SKV_L2_KEEP_PCT
+#define SKV_L2_KEEP_PCT 20
 #endif
 // Start-up offset between the compute warps of one scheduler (nanoseconds per column group).
 #ifndef SKV_STAGGER_NS
@@ -396,6 +418,11 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         tma_load_2d(base + L::kQOff + s * (L::kQBytes / L::kSub), &map_q, bars + 8 * kBarQ, s * 64, q_row0);
       int issued = 0;
       const int n_load = PASS == 1 ? 2 * n_my : n_my;      // 128-key tiles this CTA loads
+      // Pass 2 sweeps backward and meets first the tiles pass 1 read last: pass 1 asks L2 to keep
+      // the last SKV_L2_KEEP_PCT percent of its segment and lets the rest stream through; pass 2
+      // never needs a line again.
+      const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
+      const int keep_from = PASS == 1 ? n_load - (n_load * SKV_L2_KEEP_PCT) / 100 : n_load;
       for (int t = 0; t < n_load; ++t) {
         const int s = t % kStages;
         const uint32_t ph = (uint32_t)(t / kStages) & 1u;
@@ -404,9 +431,14 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         // a tile may reach beyond the sequence's last key (into zero fill, or into the next
         // sequence of a packed batch): the causal mask discards those keys
         const int tile = PASS == 1 ? 2 * t_lo + t : tile_of(t);
-        for (int c = 0; c < L::kSub; ++c)
-          tma_load_3d(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
-                      c * 64, key0 + tile * kKeyTile, g);
+        for (int c = 0; c < L::kSub; ++c) {
+          if (SKV_L2_KEEP_PCT > 0)
+            tma_load_3d_hint(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
+                             c * 64, key0 + tile * kKeyTile, g, t >= keep_from ? pol_keep : pol_stream);
+          else
+            tma_load_3d(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
+                        c * 64, key0 + tile * kKeyTile, g);
+        }
         ++issued;
       }
       // drain: every copy this thread issued must have landed before the CTA may exit
