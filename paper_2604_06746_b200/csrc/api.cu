@@ -141,7 +141,6 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
   a.n_keys = n_keys; a.scale = scale;
   a.batch = 1; a.total_keys = n_keys; a.cu_seqlens = nullptr;
-  a.group0 = 0; a.n_groups = cfg.n_kv_heads;
   a.cols = head_cols_out ? head_cols_out : c.ws.cols;
   a.col_stride = head_cols_out ? (long long)n_keys : (long long)c.n_pad;
 
@@ -149,27 +148,14 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
                       tc_supported(c, a);
   int parts = 0;
   cudaError_t e;
-#ifndef SKV_GROUP_CHUNK
-#define SKV_GROUP_CHUNK 0
-#endif
-  if (use_tc && SKV_GROUP_CHUNK > 0) {
-    // both passes of a few KV groups at a time: their K stays in L2 between the passes
-    for (int g0 = 0; g0 < cfg.n_kv_heads; g0 += SKV_GROUP_CHUNK) {
-      a.group0 = g0;
-      a.n_groups = cfg.n_kv_heads - g0 < SKV_GROUP_CHUNK ? cfg.n_kv_heads - g0 : SKV_GROUP_CHUNK;
-      if (launch_score_tc(c, a, &parts, 1, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
-      if (launch_score_tc(c, a, &parts, 2, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
-    }
-  } else {
-    e = use_tc ? launch_score_tc(c, a, &parts, 1, st) : launch_score_simt(c, a, &parts, 1, st);
-    if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
-    if (!use_tc) {
-      e = launch_finalize_rows(c, parts, st);
-      if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
-    }
-    e = use_tc ? launch_score_tc(c, a, &parts, 2, st) : launch_score_simt(c, a, &parts, 2, st);
+  e = use_tc ? launch_score_tc(c, a, &parts, 1, st) : launch_score_simt(c, a, &parts, 1, st);
+  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  if (!use_tc) {
+    e = launch_finalize_rows(c, parts, st);
     if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
   }
+  e = use_tc ? launch_score_tc(c, a, &parts, 2, st) : launch_score_simt(c, a, &parts, 2, st);
+  if (e != cudaSuccess) return STRUCTKV_ERR_CUDA;
   e = launch_reduce_finish(c, a.cols, a.col_stride, n_keys, lambda, s_out, c_inout,
                            !(flags & STRUCTKV_FLAG_NO_HEAD_STATS), metrics_out, st);
   return e == cudaSuccess ? STRUCTKV_OK : STRUCTKV_ERR_CUDA;
@@ -241,7 +227,6 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   a.q = q_window; a.k = k;
   a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
   a.n_keys = 0; a.batch = batch; a.total_keys = total; a.cu_seqlens = cu_seqlens;
-  a.group0 = 0; a.n_groups = cfg.n_kv_heads;
   a.scale = scale;
   a.cols = head_cols_out ? head_cols_out : bw.cols;
   a.col_stride = head_cols_out ? (long long)total : (long long)align_up((size_t)total, kKeyTile);

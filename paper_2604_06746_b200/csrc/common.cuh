@@ -54,7 +54,6 @@ struct ScoreArgs {
   int batch;                // sequences in the call (1 for a plain call)
   int total_keys;           // rows of K along the token axis: n_keys, or cu_seqlens[batch]
   const int* cu_seqlens;    // host, [batch + 1] first key of every sequence in the packed K; NULL = plain call
-  int group0, n_groups;     // KV groups this launch covers: [group0, group0 + n_groups)
   float scale;
   float* cols;              // [H][col_stride] pooled per-head attention (output of pass 2)
   long long col_stride;

@@ -40,7 +40,6 @@ struct SeqDesc { int key0, n_keys, cta0, segs; };
 
 struct TcParams {
   int window, group, rows_pg, rows_pg_pad, rows_pad, n_rb;
-  int group0;                          // first KV group of this launch
   int n_seq;                           // sequences in this launch
   int q_rows;                          // score rows of one sequence in the Q tensor (H * w)
   long long rows_all;                  // n_seq * rows_pad: stride between segments in row_part
@@ -367,7 +366,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   const int n_keys = p.seq[sq].n_keys, key0 = p.seq[sq].key0, segs = p.seq[sq].segs;
   const int cta = (int)blockIdx.x - p.seq[sq].cta0;
   const int unit = cta / segs, seg = cta - unit * segs;
-  const int g = p.group0 + unit / p.n_rb, rb = unit % p.n_rb;
+  const int g = unit / p.n_rb, rb = unit - g * p.n_rb;
   const size_t row_base = (size_t)sq * p.rows_pad + (size_t)g * p.rows_pg_pad + rb * kRowBlock;
   // Pass 1 walks its segment in pairs of key tiles (256 keys per MMA), pass 2 in single tiles.
   const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
@@ -996,8 +995,7 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   // The CTAs of the grid (about one per SM) are shared out over the sequences in proportion to
   // their lengths; every (KV group, row block) unit of a sequence gets the same number of key
   // segments, at least one, at most one per pair of key tiles.
-  const int units = a.n_groups * p.n_rb;
-  p.group0 = a.group0;
+  const int units = ctx.cfg.n_kv_heads * p.n_rb;
   int grid = 0, max_segs = 0;
   for (int b = 0; b < a.batch; ++b) {
     const int key0 = a.cu_seqlens ? a.cu_seqlens[b] : 0;
