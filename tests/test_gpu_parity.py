@@ -235,3 +235,27 @@ def test_batched_head_statistics_equal_the_per_layer_ones(mods, cuda_device):
         outs.append((pf.metrics.clone(), pf.s_hist.clone(), pf.pivot))
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and outs[0][2] == outs[1][2]
     assert not torch.isnan(outs[0][0]).any()
+
+
+def test_near_uniform_attention_keeps_the_variance_within_tolerance(mods, cuda_device):
+    """High temperatures flatten the attention: every pooled per-head vector is close to 1/N and its
+    variance (Eq. 6) is a small difference of nearly equal numbers.  The metric must still match
+    the oracle's population variance (it is summed as squared deviations from 1/N)."""
+    binding, _ = mods
+    wl = synth.Workload("flat", 9, 3, 8, 2, 128, 6000, 64, (512,), "bf16", 0, None, hub_layers=(),
+                        temperatures=(8.0, 5.0, 12.0))
+    pl = synth.plan(wl)
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, torch.bfloat16, cuda_device)
+    for layer in range(wl.n_layers):
+        t = synth.make_layer(wl, pl, layer, device="cpu", with_v=False)
+        s = torch.zeros(wl.seq, dtype=torch.float32, device=cuda_device)
+        m = torch.zeros(3, dtype=torch.float32, device=cuda_device)
+        ctx.score_layer(t["q_win"].to(cuda_device), t["k"].to(cuda_device), t["scale"], s, m)
+        torch.cuda.synchronize()
+        o = O.score_layer(synth.to_f64(t["q_win"]), synth.to_f64(t["k"]), t["scale"])
+        assert o["variance"] < 1e-2 / wl.seq ** 2 * 100           # the regime this test is about: tiny variance
+        P.assert_scores_close(s.cpu().numpy(), o["S"], f"flat S layer {layer}")
+        for i, key in enumerate(("entropy", "sparsity", "variance")):
+            P.assert_metric_close(m[i].item(), o[key], f"flat {key} layer {layer}")
+    assert ctx.poll_device_status() == binding.OK
+    ctx.close()
