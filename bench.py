@@ -38,8 +38,10 @@ SFU_EXP_PER_CLK_PER_SM = 16      # special-function results per clock per SM (cc
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the scorer launches of one layer,
 # from an ncu capture of the current kernels; None = no capture of the current kernels exists.
-NCU_TRAFFIC_BYTES_PER_LAYER = None
-NCU_TRAFFIC_NOTE = "pending: single-pass ncu capture (caches left as the previous kernel leaves them) of the current kernels"
+NCU_TRAFFIC_BYTES_PER_LAYER = 513.0e6
+NCU_TRAFFIC_NOTE = ("dram read + write of the two tc_score launches of one layer (llama128k shape), single-metric "
+                    "ncu captures with the caches left as the previous kernel leaves them: pass 1 reads 269 MB, "
+                    "pass 2 211-217 MB (its backward sweep finds a fifth of K in L2), 15 + 15 MB written")
 
 
 def load_peaks():
@@ -286,6 +288,50 @@ def time_streamed(wl, pl, kv_budget, dev, sweeps=2):
             for k in tot:
                 tot[k] += acc[k] / sweeps
     return pf, tot
+
+
+def batch_timing(dev, reps=10):
+    """One layer of Llama-3-8B-shaped scoring for a batch of four prompts of different lengths (131072
+    tokens together), as ONE structkv_score_layer_batch call against four structkv_score_layer calls."""
+    from paper_2604_06746_b200 import binding
+    H, Hkv, d, w = 32, 8, 128, 64
+    lens = (40000, 20000, 50000, 21072)
+    cu = [0]
+    for n in lens:
+        cu.append(cu[-1] + n)
+    total, B = cu[-1], len(lens)
+    g = torch.Generator(device=dev)
+    g.manual_seed(123)
+    q = torch.randn((B, H, w, d), generator=g, device=dev).to(torch.bfloat16)
+    k = torch.randn((Hkv, total, d), generator=g, device=dev).to(torch.bfloat16)
+    ctx = binding.Context(H, Hkv, d, w, max(lens), torch.bfloat16, dev)
+    ws = ctx.batch_workspace(B, total)
+    s = torch.zeros(total, dtype=torch.float32, device=dev)
+    m = torch.zeros((B, 3), dtype=torch.float32, device=dev)
+    scale = 1.0 / math.sqrt(d)
+
+    def batched():
+        ctx.score_layer_batch(q, k, cu, scale, s, m, ws)
+
+    def separate():
+        for b in range(B):
+            ctx.score_layer(q[b], k[:, cu[b]:cu[b + 1]], scale, s[cu[b]:cu[b + 1]], m[b])
+
+    out = {}
+    for name, fn in (("one_batched_call_us", batched), ("four_separate_calls_us", separate)):
+        fn()
+        torch.cuda.synchronize()
+        a, b_ = ev(), ev()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b_.record()
+        torch.cuda.synchronize()
+        out[name] = a.elapsed_time(b_) * 1e3 / reps
+    out["prompt_lengths"] = list(lens)
+    assert ctx.poll_device_status() == binding.OK
+    ctx.close()
+    return out
 
 
 def scorer_roofline(wl, score_ms_per_step, peaks, sm_mhz):
@@ -675,6 +721,8 @@ def main():
                  "mass_recovery_us": ex[1].elapsed_time(ex[2]) * 1e3 / reps,
                  "note": "back-to-back launches from Python; a floor of a few us per call is host launch cost",
                  "mass_recovery_of_i_struct_min_over_layers": float(rec.min().item())}
+    if wl.dtype == "bf16" and rank == 0:
+        next_rows["batched_prompts_one_layer"] = batch_timing(dev)
     pivot_timed = pf.pivot
     e2e = None if args.no_e2e else measure_e2e(res, dev, args.e2e_steps, world)
     assert pf.ctx.poll_device_status() == binding.OK
