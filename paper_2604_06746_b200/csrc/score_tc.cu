@@ -251,23 +251,9 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
   unpack2(x, x0, x1);
   return pack2(fast_exp2(x0), fast_exp2(x1));
 }
-// Scalar form of the same polynomial (pass 1).
-[[maybe_unused]] __device__ __forceinline__ float exp2_poly1(float x) {
-  x = fminf(fmaxf(x, -125.f), 126.f);
-  const float t = x + 12582912.0f;
-  const float f = x - (t - 12582912.0f);
-  float p = fmaf(0.0551716685f, f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-// In pass 1, of every 8 consecutive elements (element pairs in the packed form) the first kPoly1
-// take the polynomial.
+// In pass 1, of every 8 consecutive element pairs the first kPoly1 take the polynomial.
 #ifndef SKV_POLY1
 #define SKV_POLY1 1
-#endif
-#ifndef SKV_PACK1
-#define SKV_PACK1 1
 #endif
 // Pass 2: subtract lse inside the MMA (one extra K-step) instead of loading it from shared memory.
 #ifndef SKV_FOLD
@@ -276,10 +262,6 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x) {
 // Percentage of a pass-1 segment (its end) that L2 is asked to keep for pass 2; 0 = no hints.
 #ifndef SKV_L2_KEEP_PCT
 #define SKV_L2_KEEP_PCT 20
-#endif
-// Start-up offset between the compute warps of one scheduler (nanoseconds per column group).
-#ifndef SKV_STAGGER_NS
-#define SKV_STAGGER_NS 0
 #endif
 constexpr int kPoly1 = SKV_POLY1;
 // In pass 2, of every 8 consecutive element pairs the first kPoly2 take the polynomial, the
@@ -538,11 +520,6 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       if (lane == 0) mbar_arrive(bars + 8 * (kBarAccEmpty + t % kAccStages));
     };
 
-    // The four compute warps of a scheduler share a lane quarter and are released by the same
-    // barrier, so without help they load, compute and load again in step, and the exponential unit
-    // idles whenever all of them wait for tensor memory.  A start-up offset per column group
-    // spreads their phases; in steady state nothing brings them back in step.
-    if (SKV_STAGGER_NS > 0 && sub > 0) __nanosleep((unsigned)(sub * SKV_STAGGER_NS));
     if (PASS == 1) {
       // A unit's accumulator holds one 128-row half of the block x the pair's 256 keys.  This
       // thread owns row (quarter * 32 + lane) of BOTH halves (units alternate between them) and
@@ -557,7 +534,6 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible;
       // of every 8 elements the first kPoly1 are exponentiated on the FMA pipe
       auto accumulate = [&](RowStat& r) {
-#if SKV_PACK1
         // packed fp32: one instruction for two elements wherever the operation is not the exponential
         const uint64_t nref2 = pack2(-r.ref, -r.ref);
         uint64_t Z2 = pack2(r.Z, 0.f), U2 = pack2(r.U, 0.f);
@@ -580,15 +556,6 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         r.Z = a + b;
         unpack2(U2, a, b);
         r.U = a + b;
-#else
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float x = fmaf(v[e], p.c2, -r.ref);
-          const float pr = ((e & 7) < kPoly1) ? exp2_poly1(x) : fast_exp2(x);
-          r.Z += pr;
-          r.U = fmaf(pr, x, r.U);
-        }
-#endif
       };
       // same with the causal mask, moving the reference up to the chunk maximum first
       // (v[0] is key jb); works from registers, so the accumulator is not needed again
