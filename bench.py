@@ -180,9 +180,12 @@ class Resident:
         self.wl, self.kv_budget, self.st_budget = wl, kv_budget, wl.struct_budget(kv_budget)
         self.layers = [synth.make_layer(wl, pl, l, device=dev) for l in range(wl.n_layers)]
         self.hidden, self.positions = synth.make_hidden(wl, device=dev)
+        # every layer's Q and K are resident and complete before any step starts (the steps are
+        # bracketed by synchronisations), which is what STRUCTKV_FLAG_INPUTS_READY asks of the caller
+        from paper_2604_06746_b200 import binding
         self.pf = pipeline.Prefill(wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq,
                                    kv_budget, self.st_budget, synth.torch_dtype(wl.dtype),
-                                   hidden_dim=wl.hidden_dim, device=dev, flags=flags)
+                                   hidden_dim=wl.hidden_dim, device=dev, flags=flags | binding.FLAG_INPUTS_READY)
 
     def step(self, timed):
         pf, layers = self.pf, self.layers

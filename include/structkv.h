@@ -49,6 +49,13 @@ typedef enum { STRUCTKV_BF16 = 0, STRUCTKV_FP32 = 1 } structkv_dtype;
 /* Flags of structkv_score_layer. */
 #define STRUCTKV_FLAG_NO_HEAD_STATS 1u /* skip Eq. 5-6: metrics_out[1..2] are written as NaN */
 #define STRUCTKV_FLAG_FORCE_SIMT 2u    /* use the CUDA-core scorer even where the tensor-core one applies */
+/* The caller vouches that q_window and k are complete and visible to the device before the call
+ * is enqueued: no kernel still in flight on `stream` writes them (they were written before an
+ * earlier synchronisation, or on another stream joined through an event).  The first scorer
+ * pass then starts reading them while the kernels enqueued before it (the previous layer's
+ * column reduction) are still draining; results are identical.  Without the flag the pass
+ * waits for everything enqueued before it, as any kernel on a stream does. */
+#define STRUCTKV_FLAG_INPUTS_READY 4u
 
 typedef struct {
   int n_q_heads;        /* H, a multiple of n_kv_heads */
@@ -133,7 +140,7 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
  *   c_inout       device, [total] fp32 or NULL: C <- lambda*C + S, packed.
  *   head_cols_out device, [H, total] fp32 or NULL.
  *   metrics_out   device, [batch, 3] fp32: {entropy, sparsity, variance} of every prompt.
- *   flags         STRUCTKV_FLAG_NO_HEAD_STATS or 0.
+ *   flags         STRUCTKV_FLAG_NO_HEAD_STATS, STRUCTKV_FLAG_INPUTS_READY or 0.
  *   batch_workspace  device, 256-byte aligned, at least
  *                 structkv_batch_workspace_bytes(cfg, batch, total) bytes, caller-owned; calls that
  *                 share it must be ordered by the caller.

@@ -27,6 +27,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 BF16, FP32 = 0, 1
 FLAG_NO_HEAD_STATS = 1
 FLAG_FORCE_SIMT = 2
+FLAG_INPUTS_READY = 4
 
 
 class Config(ctypes.Structure):

@@ -133,7 +133,8 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   if (((uintptr_t)s_out % 4) || ((uintptr_t)metrics_out % 4) || ((uintptr_t)c_inout % 4) ||
       ((uintptr_t)head_cols_out % 4))
     return STRUCTKV_ERR_INVALID_ARG;
-  if (flags & ~(STRUCTKV_FLAG_NO_HEAD_STATS | STRUCTKV_FLAG_FORCE_SIMT)) return STRUCTKV_ERR_INVALID_ARG;
+  if (flags & ~(STRUCTKV_FLAG_NO_HEAD_STATS | STRUCTKV_FLAG_FORCE_SIMT | STRUCTKV_FLAG_INPUTS_READY))
+    return STRUCTKV_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
 
   ScoreArgs a;
@@ -141,6 +142,7 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
   a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
   a.n_keys = n_keys; a.scale = scale;
   a.batch = 1; a.total_keys = n_keys; a.cu_seqlens = nullptr;
+  a.inputs_ready = (flags & STRUCTKV_FLAG_INPUTS_READY) != 0;
   a.cols = head_cols_out ? head_cols_out : c.ws.cols;
   a.col_stride = head_cols_out ? (long long)n_keys : (long long)c.n_pad;
 
@@ -211,7 +213,7 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   if (((uintptr_t)q_window % 16) || ((uintptr_t)k % 16)) return STRUCTKV_ERR_INVALID_ARG;
   if (k_stride_token < cfg.head_dim || k_stride_head < 0) return STRUCTKV_ERR_INVALID_ARG;
   if ((k_stride_token * 2) % 16 || (k_stride_head * 2) % 16) return STRUCTKV_ERR_INVALID_ARG;
-  if (flags & ~STRUCTKV_FLAG_NO_HEAD_STATS) return STRUCTKV_ERR_INVALID_ARG;
+  if (flags & ~(STRUCTKV_FLAG_NO_HEAD_STATS | STRUCTKV_FLAG_INPUTS_READY)) return STRUCTKV_ERR_INVALID_ARG;
   const size_t need = carve_batch(cfg, batch, total, nullptr).bytes;
   if (!batch_workspace || batch_workspace_bytes < need || ((uintptr_t)batch_workspace % 256) != 0)
     return STRUCTKV_ERR_WORKSPACE;
@@ -228,6 +230,7 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
   a.n_keys = 0; a.batch = batch; a.total_keys = total; a.cu_seqlens = cu_seqlens;
   a.scale = scale;
+  a.inputs_ready = (flags & STRUCTKV_FLAG_INPUTS_READY) != 0;
   a.cols = head_cols_out ? head_cols_out : bw.cols;
   a.col_stride = head_cols_out ? (long long)total : (long long)align_up((size_t)total, kKeyTile);
   // only the tensor-core scorer handles packed batches

@@ -55,6 +55,7 @@ struct ScoreArgs {
   int total_keys;           // rows of K along the token axis: n_keys, or cu_seqlens[batch]
   const int* cu_seqlens;    // host, [batch + 1] first key of every sequence in the packed K; NULL = plain call
   float scale;
+  bool inputs_ready = false; // q and k are complete and visible: nothing in flight on the stream writes them
   float* cols;              // [H][col_stride] pooled per-head attention (output of pass 2)
   long long col_stride;
 };

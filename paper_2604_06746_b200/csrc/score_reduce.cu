@@ -158,15 +158,46 @@ reduce_finish(const float* __restrict__ cols, long long col_stride, int H, int n
 constexpr int kHsCluster = 8;      // CTAs per (layer, head) when few vectors are in flight (one layer at a time)
 constexpr int kHsThreads = 1024;
 constexpr int kHsBins = 2048;
-constexpr int kHsCopies = 8;      // each bin is kept 8 times (lane & 7) so that a warp's hits on one bin spread
+// each bin is kept several times (lane & (copies - 1)) so that a warp's hits on one bin spread: 8 copies
+// where a cluster shares a vector (two CTAs per SM), 16 where one CTA sweeps a whole vector (a lane
+// then shares its banks with one other lane only)
+__host__ __device__ constexpr int hs_copies(int cl) { return cl == 1 ? 16 : 8; }
 constexpr int kHsItems = 16;      // entries per thread kept in registers between the sweeps
 
-// Shared memory of head_stats: hist[kHsBins][kHsCopies] | merged[2][kHsBins] (dynamic, 80 KB).
+// Applies f to a[lo .. hi) once each, kHsThreads threads together: 16-byte loads, four of them in
+// flight per thread, scalar accesses only for the unaligned ends.  The order in which a thread
+// meets its entries is fixed.
+template <class F>
+__device__ __forceinline__ void sweep_from_memory(const float* __restrict__ a, int lo, int hi, int tid, F f) {
+  const int mis = (int)((reinterpret_cast<uintptr_t>(a + lo) >> 2) & 3u);
+  const int n_head = min(hi - lo, (4 - mis) & 3);
+  if (tid < n_head) f(a[lo + tid]);
+  const int b0 = lo + n_head;
+  const int n4 = (hi - b0) >> 2;
+  const float4* a4 = reinterpret_cast<const float4*>(a + b0);
+  int i = tid;
+  for (; i + 3 * kHsThreads < n4; i += 4 * kHsThreads) {
+    const float4 v0 = a4[i], v1 = a4[i + kHsThreads], v2 = a4[i + 2 * kHsThreads], v3 = a4[i + 3 * kHsThreads];
+    f(v0.x); f(v0.y); f(v0.z); f(v0.w);
+    f(v1.x); f(v1.y); f(v1.z); f(v1.w);
+    f(v2.x); f(v2.y); f(v2.z); f(v2.w);
+    f(v3.x); f(v3.y); f(v3.z); f(v3.w);
+  }
+  for (; i < n4; i += kHsThreads) {
+    const float4 v = a4[i];
+    f(v.x); f(v.y); f(v.z); f(v.w);
+  }
+  const int t0 = b0 + 4 * n4;
+  if (t0 + tid < hi) f(a[t0 + tid]);
+}
+
+// Shared memory of head_stats: hist[kHsBins][copies] | merged[2][kHsBins] (dynamic, 80 or 144 KB).
 template <int CL>     // CTAs that share one (layer, head) vector: kHsCluster, or 1 when a batch of layers fills the GPU
 __global__ void __launch_bounds__(kHsThreads)
 head_stats(const float* __restrict__ cols, long long layer_stride, long long col_stride, int H, int n,
            int k_rho, float* __restrict__ head_part) {
   extern __shared__ unsigned hs_smem[];
+  constexpr int kHsCopies = hs_copies(CL);
   unsigned* hist = hs_smem;                          // this CTA's counts, kHsCopies per bin
   unsigned* merged = hs_smem + kHsBins * kHsCopies;  // cluster-wide counts of the two levels (CTA 0's copy counts)
   __shared__ float red[33];
@@ -190,7 +221,7 @@ head_stats(const float* __restrict__ cols, long long layer_stride, long long col
     for (int b = tid; b < kHsBins; b += kHsThreads) {
       unsigned c = 0;
 #pragma unroll
-      for (int k = 0; k < kHsCopies; ++k) c += hist[b * kHsCopies + k];
+      for (int k = 0; k < kHsCopies; ++k) c += hist[b * kHsCopies + ((k + tid) & (kHsCopies - 1))];   // rotated: no bank conflicts
       if (c) atomicAdd(&merged0[level * kHsBins + b], c);
     }
   };
@@ -217,12 +248,11 @@ head_stats(const float* __restrict__ cols, long long layer_stride, long long col
         atomicAdd(&hist[((__float_as_uint(reg[e]) >> 20) & 0x7ffu) * kHsCopies + copy], 1u);
       }
   } else {
-    for (int j = lo + tid; j < hi; j += kHsThreads) {
-      const float v = a[j];
+    sweep_from_memory(a, lo, hi, tid, [&](float v) {
       const float dv = v - mean;
       sq = fmaf(dv, dv, sq);
       atomicAdd(&hist[((__float_as_uint(v) >> 20) & 0x7ffu) * kHsCopies + copy], 1u);
-    }
+    });
   }
   __syncthreads();
   push(0);
@@ -245,7 +275,7 @@ head_stats(const float* __restrict__ cols, long long layer_stride, long long col
     for (int e = 0; e < kHsItems; ++e)
       if (reg[e] >= 0.f) second(reg[e]);
   } else {
-    for (int j = lo + tid; j < hi; j += kHsThreads) second(a[j]);
+    sweep_from_memory(a, lo, hi, tid, second);
   }
   __syncthreads();
   push(1);
@@ -319,7 +349,7 @@ cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st) {
 template <int CL>
 static cudaError_t launch_head_stats_cl(const float* cols, long long layer_stride, long long col_stride,
                                         int n_layers, int H, int n, int k_rho, float* head_part, cudaStream_t st) {
-  const int smem = (kHsBins * kHsCopies + 2 * kHsBins) * (int)sizeof(unsigned);
+  const int smem = (kHsBins * hs_copies(CL) + 2 * kHsBins) * (int)sizeof(unsigned);
   cudaError_t e = cudaFuncSetAttribute(head_stats<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};

@@ -47,6 +47,7 @@ struct TcParams {
   float c2;                            // scale * log2(e)
   float inv_c2;                        // 1 / c2, or 0 when the fold of -lse into the MMA is off
   int fold;                            // pass 2: the accumulator already holds q.k - lse / c2
+  int inputs_ready;                    // pass 1: Q and K are complete and visible, no kernel in flight writes them
   float4* row_part;                    // pass 1 out, pass 2 in: [segs][n_seq][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): [n_seq][rows_pad] entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride], sequence b at column key0_b
@@ -388,7 +389,10 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   // so pass 2 (whose producer warps read K and Q without waiting) never runs ahead of the
   // kernel that precedes pass 1.  In pass 2 only the compute warps depend on pass 1 (the row
   // statistics): the loads of K and Q and the MMAs start at once.
-  if (PASS == 1) pdl_wait();
+  // Where the caller vouches for Q and K (inputs_ready), pass 1 starts at once as well and only
+  // its stores of the row statistics wait for the kernels before it; pass 2 still cannot begin
+  // its own stores before those kernels are done, because pass 1 cannot complete earlier.
+  if (PASS == 1 && !p.inputs_ready) pdl_wait();
   pdl_trigger();
 
   if (warp == 0) {
@@ -620,6 +624,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       // each to the largest reference M, Z = sum_c 2^(ref_c - M) Z_c,
       // U = sum_c 2^(ref_c - M) (U_c + (ref_c - M) Z_c).
       float4* part_s = reinterpret_cast<float4*>(sm + L::kMergeOff);
+      // the previous layer's pass 2 may still be reading the row statistics this pass overwrites
+      if (p.inputs_ready) pdl_wait();
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf)
         part_s[sub * kRowBlock + hf * 128 + row_lo] = make_float4(st[hf].ref, st[hf].Z, st[hf].U, 0.f);
@@ -979,6 +985,7 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.c2 = a.scale * kLog2e;
   // the fold needs a finite lse / c2 (a zero scale keeps the plain form)
   p.fold = (SKV_FOLD != 0) && pass == 2 && fabsf(p.c2) > 1e-20f ? 1 : 0;
+  p.inputs_ready = a.inputs_ready ? 1 : 0;
   p.inv_c2 = p.fold ? 1.0f / p.c2 : 0.f;
   p.row_part = ctx.ws.row_part;
   p.row_ent = ctx.ws.row_ent;

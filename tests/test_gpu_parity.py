@@ -259,3 +259,42 @@ def test_near_uniform_attention_keeps_the_variance_within_tolerance(mods, cuda_d
             P.assert_metric_close(m[i].item(), o[key], f"flat {key} layer {layer}")
     assert ctx.poll_device_status() == binding.OK
     ctx.close()
+
+
+def test_early_start_of_the_first_pass_changes_no_bit(mods, cuda_device):
+    """With STRUCTKV_FLAG_INPUTS_READY the first scorer pass of a layer starts while the previous
+    layer's column reduction is still running (its inputs are vouched for by the caller, here by a
+    synchronisation); every output must equal the unflagged run bit for bit, on a chain of layers
+    long enough for the passes of neighbouring layers to overlap."""
+    binding, pipeline = mods
+    wl = synth.WORKLOADS["llama32k"].scaled(9000 + 41, n_layers=6, n_hubs=8, budgets=(400,))
+    pl = synth.plan(wl)
+    layers = gpu_layers(wl, pl, cuda_device)
+    torch.cuda.synchronize()
+    outs = []
+    for flags in (0, binding.FLAG_INPUTS_READY, binding.FLAG_INPUTS_READY):
+        pf = pipeline.Prefill(wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq,
+                              wl.budget, wl.struct_budget(), torch.bfloat16, device=cuda_device, flags=flags)
+        torch.cuda.synchronize()
+        for _ in range(3):                       # repeated sweeps: layer 0 follows layer L-1 back to back
+            for l, t in enumerate(layers):
+                pf.score(l, t["q_win"], t["k"], t["scale"])
+        pf.detect_and_select()
+        torch.cuda.synchronize()
+        assert pf.ctx.poll_device_status() == binding.OK
+        outs.append((pf.metrics.clone(), pf.s_hist.clone(), pf.c_running.clone(), pf.i_kv.clone(), pf.pivot))
+    for o in outs[1:]:
+        assert all(torch.equal(a, b) for a, b in zip(outs[0][:4], o[:4])) and o[4] == outs[0][4]
+    # the batch entry point takes the flag too; any other bit is refused
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, torch.bfloat16, cuda_device)
+    t = layers[0]
+    s1, s2 = (torch.zeros(wl.seq, device=cuda_device) for _ in range(2))
+    m1, m2 = torch.zeros(3, device=cuda_device), torch.zeros((1, 3), device=cuda_device)
+    ctx.score_layer(t["q_win"], t["k"], t["scale"], s1, m1, flags=binding.FLAG_INPUTS_READY)
+    ctx.score_layer_batch(t["q_win"][None], t["k"], [0, wl.seq], t["scale"], s2, m2, ctx.batch_workspace(1, wl.seq),
+                          flags=binding.FLAG_INPUTS_READY)
+    torch.cuda.synchronize()
+    assert torch.equal(s1, s2) and torch.equal(m1, m2[0])
+    with pytest.raises(Exception):
+        ctx.score_layer(t["q_win"], t["k"], t["scale"], s1, m1, flags=8)
+    ctx.close()
