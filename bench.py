@@ -560,7 +560,7 @@ def measure_e2e(res, dev, steps, world):
 
 # ------------------------------------------------------------------------------------------------
 def run_reference(args):
-    """The reference arm of this build is the CPU oracle (the paper ships no code)."""
+    """The reference arm is the CPU oracle (the paper ships no code)."""
     from paper_2604_06746_b200 import synth
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
