@@ -96,15 +96,25 @@ def score_layer(q_win: np.ndarray, k: np.ndarray, scale: float) -> Dict[str, np.
             term = np.where(a > 0.0, a * np.log(a), 0.0)
         row_entropy[h] = -term.sum(axis=1)
     S = head_cols.sum(axis=0)
-    k_rho = max(1, N // SPARSITY_DENOMINATOR)
-    top_mass = np.sort(head_cols, axis=1)[:, ::-1][:, :k_rho].sum(axis=1)
+    sparsity, variance = head_statistics(head_cols)
     return {
         "S": S,
         "head_cols": head_cols,
         "entropy": float(row_entropy.mean()),
-        "sparsity": float(top_mass.mean()),
-        "variance": float(np.var(head_cols, axis=1).mean()),
+        "sparsity": sparsity,
+        "variance": variance,
     }
+
+
+def head_statistics(head_cols: np.ndarray) -> Tuple[float, float]:
+    """Eq. 5 and Eq. 6 from the window-pooled per-head attention ``head_cols [H, N]`` (R5, R6):
+    the mean over heads of the mass of the ``floor(0.1 N)`` largest entries, and the mean over
+    heads of the population variance over the keys."""
+    head_cols = np.asarray(head_cols, dtype=np.float64)
+    N = head_cols.shape[1]
+    k_rho = max(1, N // SPARSITY_DENOMINATOR)
+    top_mass = np.sort(head_cols, axis=1)[:, ::-1][:, :k_rho].sum(axis=1)
+    return float(top_mass.mean()), float(np.var(head_cols, axis=1).mean())
 
 
 # --------------------------------------------------------------------------- Eq. 3

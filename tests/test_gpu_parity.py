@@ -298,3 +298,35 @@ def test_early_start_of_the_first_pass_changes_no_bit(mods, cuda_device):
     with pytest.raises(Exception):
         ctx.score_layer(t["q_win"], t["k"], t["scale"], s1, m1, flags=8)
     ctx.close()
+
+
+def test_batched_head_statistics_on_unaligned_vectors(mods, cuda_device):
+    """structkv_head_stats on enough vectors for the one-CTA-per-vector form, each longer than the
+    register-resident limit and starting at every 16-byte misalignment (odd length, packed rows):
+    its 16-byte memory sweeps must take the ragged ends with scalar accesses.  Eq. 5-6 against the
+    oracle, vectors with ties, zeros and a few dominant entries."""
+    binding, _ = mods
+    L, H, N = 10, 32, 20011
+    rng = np.random.default_rng(77)
+    x = rng.random((L, H, N)) ** 4
+    x[:, :, ::7] = 0.0                                   # exact zeros
+    n_tie = min(x[:, :, 5::11].shape[2], x[:, :, 6::11].shape[2])
+    x[:, :, 5:5 + 11 * n_tie:11] = x[:, :, 6:6 + 11 * n_tie:11]     # planted ties
+    hot = rng.integers(0, N, size=(L, H, 6))
+    for l in range(L):
+        for h in range(H):
+            x[l, h, hot[l, h]] += 40.0 * (1 + l)         # the top mass differs from layer to layer
+    x /= x.sum(axis=2, keepdims=True)
+    x32 = x.astype(np.float32)
+    hc = torch.from_numpy(x32).to(cuda_device)
+    m = torch.zeros((L, 3), dtype=torch.float32, device=cuda_device)
+    ctx = binding.Context(H, 8, 128, 64, N, torch.bfloat16, cuda_device)
+    ctx.head_stats(hc, m)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == binding.OK
+    got = m.cpu().numpy()
+    for l in range(L):
+        rho, var = O.head_statistics(x32[l].astype(np.float64))
+        P.assert_metric_close(got[l, 1], rho, f"sparsity of layer {l}")
+        P.assert_metric_close(got[l, 2], var, f"variance of layer {l}")
+    ctx.close()

@@ -173,3 +173,36 @@ def test_entropy_bounds_and_scale_sign():
     k1 = np.zeros((1, 9, 3)); k1[0, 4, 1] = 3.0; k1[0, 2, 1] = -3.0
     S = O.score_layer(q1, k1, 1.0)["S"]
     assert S.argmax() == 4 and S.argmin() == 2
+
+
+def test_head_statistics_closed_forms_and_brute_force():
+    """Eq. 5-6 on pooled vectors given directly: uniform vectors (top mass k/N, zero variance),
+    one-hot vectors (top mass 1, variance (1/N)(1 - 1/N)), a two-level vector worked by hand, and a
+    pure-Python selection of the largest entries."""
+    N = 50                                                       # k_rho = 5
+    rho, var = O.head_statistics(np.full((3, N), 1.0 / N))
+    assert rho == pytest.approx(5.0 / N, rel=1e-14) and var == pytest.approx(0.0, abs=1e-30)
+    one_hot = np.zeros((2, N))
+    one_hot[0, 7] = one_hot[1, 49] = 1.0
+    rho, var = O.head_statistics(one_hot)
+    assert rho == pytest.approx(1.0) and var == pytest.approx((1.0 / N) * (1.0 - 1.0 / N), rel=1e-13)
+    # 3 entries of 0.2 and 47 of 0.4 / 47: the five largest are the three big ones and two small ones
+    two = np.full((1, N), 0.4 / 47)
+    two[0, [4, 20, 33]] = 0.2
+    rho, var = O.head_statistics(two)
+    assert rho == pytest.approx(0.6 + 2 * 0.4 / 47, rel=1e-13)
+    assert var == pytest.approx((3 * 0.2 ** 2 + 47 * (0.4 / 47) ** 2) / N - (1.0 / N) ** 2, rel=1e-12)
+    # heads are averaged: a uniform and a one-hot head together
+    rho, var = O.head_statistics(np.stack([np.full(N, 1.0 / N), one_hot[0]]))
+    assert rho == pytest.approx(0.5 * (5.0 / N + 1.0)) and var == pytest.approx(0.5 * (1.0 / N) * (1.0 - 1.0 / N))
+    rng = np.random.default_rng(5)
+    x = rng.random((4, 37)) ** 3
+    x /= x.sum(axis=1, keepdims=True)
+    want_rho = want_var = 0.0
+    for row in x:
+        vals = sorted(row.tolist(), reverse=True)
+        want_rho += sum(vals[:3])                                # floor(0.1 * 37) = 3
+        mean = sum(row.tolist()) / 37
+        want_var += sum((v - mean) ** 2 for v in row.tolist()) / 37
+    rho, var = O.head_statistics(x)
+    assert rho == pytest.approx(want_rho / 4, rel=1e-13) and var == pytest.approx(want_var / 4, rel=1e-12)
