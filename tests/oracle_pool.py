@@ -56,9 +56,10 @@ def default_workers(bytes_per_worker: float) -> int:
 
 
 def score_layers(tasks: Iterable[Tuple[int, np.ndarray, np.ndarray, float, Optional[int]]], n_tasks: int,
-                 workers: int) -> Tuple[np.ndarray, np.ndarray]:
+                 workers: int, stack: bool = True):
     """``tasks`` yields ``(layer, q_bits, k_bits, scale, n_keys or None)``; returns the oracle's
-    ``s_hist [L, N]`` and ``metrics [L, 3]`` (layers indexed by the ``layer`` field, 0 .. L-1)."""
+    ``s_hist [L, N]`` and ``metrics [L, 3]`` (layers indexed by the ``layer`` field, 0 .. L-1).
+    With ``stack=False`` the score vectors come back as a list (tasks of different lengths)."""
     saved = {v: os.environ.get(v) for v in _THREAD_VARS}
     for v in _THREAD_VARS:                      # one compute thread per worker: the layers run side by side
         os.environ[v] = "1"
@@ -89,7 +90,7 @@ def score_layers(tasks: Iterable[Tuple[int, np.ndarray, np.ndarray, float, Optio
                 os.environ.pop(v, None)
             else:
                 os.environ[v] = old
-    return np.stack(s_hist), metrics
+    return (np.stack(s_hist) if stack else s_hist), metrics
 
 
 def assemble(s_hist: np.ndarray, metrics: np.ndarray, window: int, kv_budgets: Sequence[int],

@@ -147,3 +147,57 @@ def test_a_batch_of_one_equals_the_plain_call(cuda_device):
     assert bad(ctx._h, q.data_ptr(), k.data_ptr(), k.stride(0), k.stride(1), cu, 1, 1.0, 0.9, s2.data_ptr(), None,
                None, m2.data_ptr(), 0, s2.data_ptr(), 16, None) == binding.ERR_WORKSPACE
     ctx.close()
+
+
+def test_batched_scoring_at_the_size_the_bench_times(cuda_device):
+    """Four Llama-3-8B-shaped prompts of 40000 + 20000 + 50000 + 21072 tokens (131072 together: the
+    batch bench.py times) scored by one structkv_score_layer_batch call per layer: every prompt's S,
+    entropy, sparsity and variance against the oracle on that prompt alone (its layers run in worker
+    processes), and the batch's outputs against four plain calls."""
+    from paper_2604_06746_b200 import binding
+    from tests import oracle_pool
+    dev = cuda_device
+    H, Hkv, d, w = 32, 8, 128, 64
+    lens = (40000, 20000, 50000, 21072)
+    n_layers = 2
+    cu = [0]
+    for n in lens:
+        cu.append(cu[-1] + n)
+    total, B = cu[-1], len(lens)
+    base = synth.WORKLOADS["llama128k"]
+    wls = [dataclasses.replace(base.scaled(n, n_layers=n_layers, n_hubs=32, budgets=(1024,)), index=60 + 3 * b)
+           for b, n in enumerate(lens)]
+    plans = [synth.plan(x) for x in wls]
+    ctx = binding.Context(H, Hkv, d, w, max(lens), torch.bfloat16, dev)
+    ws = ctx.batch_workspace(B, total)
+    s_b = torch.zeros((n_layers, total), dtype=torch.float32, device=dev)
+    m_b = torch.zeros((n_layers, B, 3), dtype=torch.float32, device=dev)
+    s_1 = torch.zeros_like(s_b)
+    m_1 = torch.zeros_like(m_b)
+    tasks = []
+    for l in range(n_layers):
+        per = [synth.make_layer(x, pl, l, device="cpu", with_v=False) for x, pl in zip(wls, plans)]
+        scale = per[0]["scale"]
+        for b in range(1, B):                                # one logit scale per call: fold the others into q
+            per[b]["q_win"] = (per[b]["q_win"].float() * (per[b]["scale"] / scale)).to(torch.bfloat16)
+        q = torch.stack([t["q_win"] for t in per]).to(dev)
+        k = torch.cat([t["k"] for t in per], dim=1).to(dev).contiguous()
+        ctx.score_layer_batch(q, k, cu, scale, s_b[l], m_b[l], ws)
+        for b in range(B):
+            ctx.score_layer(q[b], k[:, cu[b]:cu[b + 1]], scale, s_1[l, cu[b]:cu[b + 1]], m_1[l, b])
+            tasks.append((l * B + b, oracle_pool.bits_of(per[b]["q_win"]), oracle_pool.bits_of(per[b]["k"]), scale, None))
+        torch.cuda.synchronize()
+    assert ctx.poll_device_status() == binding.OK
+    # a prompt's keys are cut into fewer segments inside a batch than alone, so the statistics are
+    # summed in another order: equal to rounding, not bit for bit
+    assert torch.allclose(s_b, s_1, rtol=1e-4, atol=1e-10) and torch.allclose(m_b, m_1, rtol=1e-4, atol=0.0)
+    workers = oracle_pool.default_workers(8.0 * H * max(lens) * 3)
+    o_s, o_m = oracle_pool.score_layers(iter(tasks), len(tasks), workers, stack=False)
+    g_s, g_m = s_b.cpu().numpy(), m_b.cpu().numpy()
+    for l in range(n_layers):
+        for b in range(B):
+            i = l * B + b
+            P.assert_scores_close(g_s[l, cu[b]:cu[b + 1]], o_s[i], f"layer {l} prompt {b} S")
+            for c in range(3):
+                P.assert_metric_close(g_m[l, b, c], o_m[i, c], f"layer {l} prompt {b} metric {c}")
+    ctx.close()
