@@ -13,8 +13,9 @@ constexpr int kKeyTile = 128;        // keys per tile in every scorer
 constexpr int kMaxParts = 160;       // upper bound on key segments per score row
 constexpr int kRowBlock = 256;       // score rows (head, window row) per tensor-core row block
 constexpr int kMaxBatch = 32;        // sequences one batched scoring call may hold
-constexpr int kMaxStatLayers = 128;
-constexpr int kMaxGatherLayers = 128; // layers one multi-layer gather may cover (their pointers are a kernel argument)  // layers one batched head-statistics call may cover
+constexpr int kMaxStatLayers = 128;   // layers one batched head-statistics call may cover
+constexpr int kMaxGatherLayers = 128; // layers one multi-layer gather may cover (their pointers are a kernel argument)
+constexpr int kQueueUnits = 256;      // (KV group, row block) units of one sequence the scorer's work queue can hold
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -26,6 +27,10 @@ struct Workspace {
   float* row_ent;       // [rows_pad] entropy of each score row (nats)
   float* cols;          // [H][n_pad] pooled per-head attention when the caller passes none
   float* head_part;     // [kMaxStatLayers][H][4] per-(layer, head) {sum of squared deviations from 1/n, top-k mass}
+  // [kQueueUnits] ticket counters of the tensor-core scorer's second pass, one per (KV group,
+  // row block); zero when the context is created, never reset: every launch advances them by a
+  // known amount (queue_base in Ctx follows)
+  unsigned long long* queue;
   size_t bytes;
 };
 
@@ -38,6 +43,8 @@ struct Ctx {
   int rows_pad;         // rows per KV group padded to kRowBlock, times H_kv
   int n_pad;            // max_seq rounded up to kKeyTile
   void* tc;             // tensor-core scorer state (tensor maps), owned by score_tc.cu
+  unsigned long long queue_base = 0;        // first ticket of the next launch of the scorer's second pass (units on full row blocks)
+  unsigned long long queue_base_last = 0;   // the same for the units on a KV group's last row block
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

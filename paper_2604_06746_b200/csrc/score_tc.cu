@@ -10,11 +10,16 @@
 // neighbouring stages of the K ring form one 256-key operand), pass 2 one 128-key tile with the
 // whole 256-row Q block.  (An N128 MMA reads as many operand bytes from shared memory per clock
 // as the SM can deliver, and slows down as soon as anything else touches shared memory.)
-// A work unit is (KV group g, row block rb of up to 256 score rows); the key range of a unit
-// is split into `segs` equal segments, one CTA each.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the
+// A work unit is (KV group g, row block rb of up to 256 score rows), served by `segs` CTAs.  In
+// pass 1 each of them owns a fixed, equal share of the unit's key-tile pairs (its partial row
+// statistics must not depend on timing); in pass 2 they draw key tiles from the unit's ticket
+// counter, so that all of them finish within one tile of each other whenever they started.
+// Warp roles: warp 0 = TMA producer (and ticket taker), warp 1 = MMA issuer (owns the
 // tensor-memory allocation), warps 2..17 = compute (four per scheduler, so that one warp's
-// tensor-memory load latency hides behind the others' arithmetic).  Pass 2 starts by merging
-// the segments' row statistics into each row's log-sum-exp (and, in segment 0, its entropy).
+// tensor-memory load latency hides behind the others' arithmetic).  Which item a K stage or an
+// accumulator holds travels with it through shared memory; an end mark follows the last item.
+// Pass 2 starts by merging the pass-1 CTAs' row statistics into each row's log-sum-exp (and, in
+// segment 0, its entropy).
 // Every wait is bounded; on expiry the CTA records STRUCTKV_ERR_TIMEOUT and stops issuing work;
 // it then waits (with a fresh bound that ignores the abort flag) for its own copies and MMAs in
 // flight, and frees tensor memory only if those MMAs are known to have retired.
@@ -34,9 +39,11 @@ constexpr int kTcThreads = 64 + kComputeThreads;   // TMA warp, MMA warp, comput
 constexpr unsigned long long kWaitCycles = 1000000000ull;   // about 0.5 s at the maximum SM clock
 constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 0 * x stays finite
 
-// One sequence of a call: its keys are rows [key0, key0 + n_keys) of the packed K, its CTAs are
-// [cta0, cta0 + units * segs) of the grid.  A plain call is a batch of one.
-struct SeqDesc { int key0, n_keys, cta0, segs; };
+// One sequence of a call: its keys are rows [key0, key0 + n_keys) of the packed K.  Every full
+// row block of a KV group is worked on by `segs` CTAs and the group's last row block by
+// `segs_last` (fewer when it holds only one 128-row half), so a group takes
+// (n_rb - 1) * segs + segs_last consecutive CTAs from cta0 on.  A plain call is a batch of one.
+struct SeqDesc { int key0, n_keys, cta0, segs, segs_last; };
 
 struct TcParams {
   int window, group, rows_pg, rows_pg_pad, rows_pad, n_rb;
@@ -48,6 +55,11 @@ struct TcParams {
   float inv_c2;                        // 1 / c2, or 0 when the fold of -lse into the MMA is off
   int fold;                            // pass 2: the accumulator already holds q.k - lse / c2
   int inputs_ready;                    // pass 1: Q and K are complete and visible, no kernel in flight writes them
+  // Work queue of pass 2: one ticket counter per (sequence, KV group, row block); a CTA draws
+  // key tiles of its unit from it until the unit has none left.  The counters only ever grow;
+  // a launch's tickets start at queue_base.
+  unsigned long long* queue;
+  unsigned long long queue_base, queue_base_last;   // units on full row blocks / on a group's last row block
   float4* row_part;                    // pass 1 out, pass 2 in: [segs][n_seq][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): [n_seq][rows_pad] entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride], sequence b at column key0_b
@@ -346,20 +358,31 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int sq = 0;                                                // the sequence this CTA works on
   while (sq + 1 < p.n_seq && (int)blockIdx.x >= p.seq[sq + 1].cta0) ++sq;
-  const int n_keys = p.seq[sq].n_keys, key0 = p.seq[sq].key0, segs = p.seq[sq].segs;
+  const int n_keys = p.seq[sq].n_keys, key0 = p.seq[sq].key0;
   const int cta = (int)blockIdx.x - p.seq[sq].cta0;
-  const int unit = cta / segs, seg = cta - unit * segs;
-  const int g = unit / p.n_rb, rb = unit - g * p.n_rb;
+  const int per_group = (p.n_rb - 1) * p.seq[sq].segs + p.seq[sq].segs_last;
+  const int g = cta / per_group, in_group = cta - g * per_group;
+  const int rb = min(in_group / p.seq[sq].segs, p.n_rb - 1);
+  const int seg = in_group - rb * p.seq[sq].segs;
+  const int segs = rb == p.n_rb - 1 ? p.seq[sq].segs_last : p.seq[sq].segs;
+  const int unit = g * p.n_rb + rb;
   const size_t row_base = (size_t)sq * p.rows_pad + (size_t)g * p.rows_pg_pad + rb * kRowBlock;
-  // Pass 1 walks its segment in pairs of key tiles (256 keys per MMA), pass 2 in single tiles.
+  // Pass 1 works on pairs of key tiles (256 keys per MMA), pass 2 on single tiles.
+  // Pass 1: CTA `seg` of a unit owns a fixed, contiguous range of pairs.  Its row statistics are
+  // partial sums over exactly that range, so the result does not depend on timing (the same
+  // inputs give the same bits).
+  // Pass 2: a tile's column sums do not depend on who computes them, so the CTAs of a unit draw
+  // tiles from the unit's ticket counter: one that starts late or runs slowly simply takes fewer,
+  // and all CTAs of a unit finish within one tile of each other.  Tiles are handed out from the
+  // end of the sequence: the tiles pass 1 touched last are the ones still in L2.
   const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
   const int n_items = PASS == 1 ? (n_tiles + 1) / 2 : n_tiles;
-  const int t_lo = (int)((long long)seg * n_items / segs);
-  const int t_hi = (int)((long long)(seg + 1) * n_items / segs);
-  const int n_my = t_hi - t_lo;
-  // Pass 1 sweeps forward, pass 2 backward: the tiles pass 1 touched last are the ones still
-  // in L2 when pass 2 starts.
-  auto tile_of = [&](int t) { return PASS == 1 ? t_lo + t : t_hi - 1 - t; };
+  const int t_lo = (int)((long long)seg * n_items / segs);          // pass 1: first pair of this CTA
+  const int n_static = (int)((long long)(seg + 1) * n_items / segs) - t_lo;
+  const int units_per_seq = p.n_rb * (p.rows_pad / p.rows_pg_pad);
+  unsigned long long* const ticket = p.queue + (size_t)sq * units_per_seq + unit;
+  int* item_s = reinterpret_cast<int*>(sm + L::kBarOff + 8 * kBarCount + 32);      // producer -> MMA issuer, per K slot
+  volatile int* unit_item = reinterpret_cast<volatile int*>(sm + L::kBarOff + 8 * kBarCount + 48);   // MMA issuer -> compute warps, per accumulator stage
   const int rows_here = min(kRowBlock, p.rows_pg - rb * kRowBlock);     // valid score rows in this block
   const int n_half = (rows_here + 127) / 128;
 
@@ -397,54 +420,91 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (lane == 0 && n_my > 0) {
+    if (lane == 0) {
+      // first ticket at once: its latency hides behind the Q load
+      unsigned long long tk = PASS == 2 ? atomicAdd(ticket, 1ull) : 0ull;
       mbar_expect_tx(bars + 8 * kBarQ, L::kQBytes);
       const int q_row0 = sq * p.q_rows + g * p.rows_pg + rb * kRowBlock;
       for (int s = 0; s < L::kSub; ++s)
         tma_load_2d(base + L::kQOff + s * (L::kQBytes / L::kSub), &map_q, bars + 8 * kBarQ, s * 64, q_row0);
-      int issued = 0;
-      const int n_load = PASS == 1 ? 2 * n_my : n_my;      // 128-key tiles this CTA loads
-      // Pass 2 sweeps backward and meets first the tiles pass 1 read last: pass 1 asks L2 to keep
-      // the last SKV_L2_KEEP_PCT percent of its segment and lets the rest stream through; pass 2
+      int issued = 0;                                      // 128-key tiles requested so far
+      bool end_marked = false;
+      // Pass 2 meets first the tiles pass 1 read last: pass 1 asks L2 to keep the last
+      // SKV_L2_KEEP_PCT percent of the sequence's keys and lets the rest stream through; pass 2
       // never needs a line again.
       const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
-      const int keep_from = PASS == 1 ? n_load - (n_load * SKV_L2_KEEP_PCT) / 100 : n_load;
-      for (int t = 0; t < n_load; ++t) {
-        const int s = t % kStages;
-        const uint32_t ph = (uint32_t)(t / kStages) & 1u;
-        if (!mbar_wait_producer(bars + 8 * (kBarEmpty + s), ph ^ 1u, abort_flag, kWaitCycles)) break;
-        mbar_expect_tx(bars + 8 * (kBarFull + s), L::kKBytes);
-        // a tile may reach beyond the sequence's last key (into zero fill, or into the next
-        // sequence of a packed batch): the causal mask discards those keys
-        const int tile = PASS == 1 ? 2 * t_lo + t : tile_of(t);
-        for (int c = 0; c < L::kSub; ++c) {
-          if (SKV_L2_KEEP_PCT > 0)
-            tma_load_3d_hint(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
-                             c * 64, key0 + tile * kKeyTile, g, t >= keep_from ? pol_keep : pol_stream);
-          else
-            tma_load_3d(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
-                        c * 64, key0 + tile * kKeyTile, g);
+      const int keep_from = PASS == 1 ? n_items - (n_items * SKV_L2_KEEP_PCT) / 100 : n_items;
+      constexpr int kPerItem = PASS == 1 ? 2 : 1;          // K stages one item occupies
+      for (int it = 0;; ++it) {
+        int item;
+        if (PASS == 1) {
+          item = it < n_static ? t_lo + it : -1;
+        } else {
+          const long long idx = (long long)(tk - (rb == p.n_rb - 1 ? p.queue_base_last : p.queue_base));
+          item = idx < (long long)n_items ? n_items - 1 - (int)idx : -1;
+          if (item >= 0) tk = atomicAdd(ticket, 1ull);     // the next ticket travels while this tile is loaded
         }
-        ++issued;
+        const int s0 = (kPerItem * it) % kStages;
+        const uint32_t ph = (uint32_t)((kPerItem * it) / kStages) & 1u;
+        if (!mbar_wait_producer(bars + 8 * (kBarEmpty + s0), ph ^ 1u, abort_flag, kWaitCycles)) break;
+        item_s[s0 / kPerItem] = item;                      // read by the MMA issuer once the stage is full
+        if (item < 0) {                                    // nothing left: an empty "full" stage says so
+          mbar_arrive(bars + 8 * (kBarFull + s0));
+          end_marked = true;
+          break;
+        }
+        bool ok = true;
+#pragma unroll
+        for (int half = 0; half < kPerItem && ok; ++half) {
+          const int s = s0 + half;
+          if (half > 0) ok = mbar_wait_producer(bars + 8 * (kBarEmpty + s), ph ^ 1u, abort_flag, kWaitCycles);
+          if (!ok) break;
+          mbar_expect_tx(bars + 8 * (kBarFull + s), L::kKBytes);
+          // a tile may reach beyond the sequence's last key (into zero fill, or into the next
+          // sequence of a packed batch): the causal mask discards those keys
+          const int tile = kPerItem * item + half;
+          for (int c = 0; c < L::kSub; ++c) {
+            if (SKV_L2_KEEP_PCT > 0)
+              tma_load_3d_hint(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
+                               c * 64, key0 + tile * kKeyTile, g, item >= keep_from ? pol_keep : pol_stream);
+            else
+              tma_load_3d(base + L::kKOff + (c * kStages + s) * L::kKSub, &map_k, bars + 8 * (kBarFull + s),
+                          c * 64, key0 + tile * kKeyTile, g);
+          }
+          ++issued;
+        }
+        if (!ok) break;
       }
-      // drain: every copy this thread issued must have landed before the CTA may exit
+      // drain: every copy this thread issued must have landed before the CTA may exit.  The end
+      // mark went into the stage of copy (issued - kStages): that copy was seen consumed before the
+      // mark was placed, and its barrier has moved on by two phases, so it is not waited for.
       mbar_drain(bars + 8 * kBarQ, 0, abort_flag);
-      for (int t = max(0, issued - kStages); t < issued; ++t)
+      for (int t = max(0, issued - kStages + (end_marked ? 1 : 0)); t < issued; ++t)
         mbar_drain(bars + 8 * (kBarFull + t % kStages), (uint32_t)(t / kStages) & 1u, abort_flag);
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0 && n_my > 0) {
+    if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(128, 256);
       const uint64_t q_desc0 = smem_desc(base + L::kQOff), k_desc0 = smem_desc(base + L::kKOff);
       bool ok = mbar_wait_producer(bars + 8 * kBarQ, 0, abort_flag, kWaitCycles);
+      // Tells the compute warps through accumulator stage `a` of unit `u` that no unit follows.
+      auto announce_end = [&](int u) {
+        const int a = u % kAccStages;
+        if (!mbar_wait_producer(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(u / kAccStages) & 1u) ^ 1u, abort_flag, kWaitCycles))
+          return;
+        unit_item[a] = -1;
+        mbar_arrive(bars + 8 * (kBarAccFull + a));
+      };
       // descriptors differ only in the start-address field (16-byte units, no carry out of it)
       if (PASS == 1) {
         // unit u = (pair, row half): A = one 128-row half of Q, B = the pair's 256 keys
-        for (int t = 0, u = 0; ok && t < n_my; ++t) {
+        for (int t = 0, u = 0; ok; ++t) {
           const int s0 = (2 * t) % kStages;
           const uint32_t ph = (uint32_t)((2 * t) / kStages) & 1u;
           if (!mbar_wait_producer(bars + 8 * (kBarFull + s0), ph, abort_flag, kWaitCycles)) break;
+          const int item = item_s[s0 / 2];
+          if (item < 0) { announce_end(u); break; }
           if (!mbar_wait_producer(bars + 8 * (kBarFull + s0 + 1), ph, abort_flag, kWaitCycles)) break;
           const uint64_t kd = k_desc0 + (uint64_t)((s0 * L::kKSub) >> 4);
           for (int hf = 0; hf < n_half; ++hf, ++u) {
@@ -461,6 +521,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
               tc_mma_bf16(tmem + a * 256, q_desc0 + (qo >> 4), kd + (ko >> 4), idesc, kk > 0);
             }
             *mma_in_flight = 1;
+            unit_item[a] = item;                       // which pair the accumulator holds
+            __threadfence_block();
             tc_commit(bars + 8 * (kBarAccFull + a));   // accumulator ready for the compute warps
           }
           if (!ok) break;
@@ -468,9 +530,11 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
           tc_commit(bars + 8 * (kBarEmpty + s0 + 1));
         }
       } else {
-        for (int t = 0; ok && t < n_my; ++t) {
+        for (int t = 0; ok; ++t) {
           const int s = t % kStages, a = t % kAccStages;
           if (!mbar_wait_producer(bars + 8 * (kBarFull + s), (uint32_t)(t / kStages) & 1u, abort_flag, kWaitCycles)) break;
+          const int item = item_s[s];
+          if (item < 0) { announce_end(t); break; }
           if (!mbar_wait_producer(bars + 8 * (kBarAccEmpty + a), ((uint32_t)(t / kAccStages) & 1u) ^ 1u, abort_flag, kWaitCycles)) break;
           tc_fence_after();
           const uint64_t kd = k_desc0 + (uint64_t)((s * L::kKSub) >> 4);
@@ -488,6 +552,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
             tc_mma_bf16(tmem + a * 256, smem_desc_k16(base + L::kMergeOff + 4096),
                         smem_desc_k16(base + L::kMergeOff + 8192), idesc, 1);
           }
+          unit_item[a] = item;                         // which tile the accumulator holds
+          __threadfence_block();
           tc_commit(bars + 8 * (kBarEmpty + s));       // K stage reusable once these MMAs have read it
           tc_commit(bars + 8 * (kBarAccFull + a));     // accumulator ready for the compute warps
         }
@@ -508,14 +574,16 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     // the first (N - w + 1) / 128 tiles are
     const int first_tail_tile = (n_keys - p.window + 1) / kKeyTile;
     float v[32];
-    // lane 0 polls the barrier for its warp (bounded); the outcome is broadcast
+    // lane 0 polls the barrier for its warp (bounded) and reads which item the accumulator
+    // holds; the outcome is broadcast: the item, -1 when the unit has no item left, -2 after an
+    // expired wait
     auto acc_full = [&](int t) {
-      int ok = 1;
-      if (lane == 0)
-        ok = mbar_wait(bars + 8 * (kBarAccFull + t % kAccStages), (uint32_t)(t / kAccStages) & 1u, abort_flag);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
+      int item = -2;
+      if (lane == 0 && mbar_wait(bars + 8 * (kBarAccFull + t % kAccStages), (uint32_t)(t / kAccStages) & 1u, abort_flag))
+        item = unit_item[t % kAccStages];
+      item = __shfl_sync(0xffffffffu, item, 0);
       tc_fence_after();
-      return ok != 0;
+      return item;
     };
     // all of this warp's loads of the tile have landed: one arrival per warp frees the accumulator
     auto acc_release = [&](int t) {
@@ -598,19 +666,20 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         }
       };
       bool live = true;
-      for (int t = 0, u = 0; live && t < n_my; ++t) {
-        const int jb = (t_lo + t) * (2 * kKeyTile) + sub * 64;
-        const bool plain = (t_lo + t) < first_tail_pair;
+      for (int t = 0, u = 0; live; ++t) {
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           if (hf < n_half && live) {
-            if (!acc_full(u)) { live = false; continue; }
+            const int item = acc_full(u);                 // the same pair for both row halves
+            if (item < 0) { live = false; continue; }
+            const int jb = item * (2 * kKeyTile) + sub * 64;
+            const bool plain = item < first_tail_pair;
             const bool warp_active = (hf * 128 + quarter * 32) < rows_here;
             const uint32_t taddr = tmem + lane_base + (uint32_t)((u % kAccStages) * 256 + sub * 64);
             if (warp_active) {
               tmem_ld32(taddr, v);
               tmem_ld_wait(v);
-              chunk(st[hf], jb, plain && t > 0);
+              chunk(st[hf], jb, plain && t > 0);          // the first pair gives the rows their reference
               tmem_ld32(taddr + 32, v);
               tmem_ld_wait(v);
             }
@@ -698,7 +767,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
           Xt = fmaf(wgt, (ref_s - M) + X_s / Z_s, Xt);
         };
         if (r < rows_here) {
-          constexpr int kBatch = 6;
+          constexpr int kBatch = 9;                      // 18 segments (one per SM share of a KV group): one round of loads
           for (int s0 = hp; s0 < parts; s0 += 2 * kBatch) {
             float4 pv[kBatch];
 #pragma unroll
@@ -809,9 +878,9 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         }
         return s;
       };
-      for (int t = 0; t < n_my; ++t) {
-        if (!acc_full(t)) break;
-        const int tile = tile_of(t);
+      for (int t = 0;; ++t) {
+        const int tile = acc_full(t);
+        if (tile < 0) break;
         const int j = tile * kKeyTile + quarter * 32 + lane;
         const bool plain = tile < first_tail_tile;
         const int i_min = j - (n_keys - p.window);        // window rows i < i_min do not see key j
@@ -932,6 +1001,8 @@ bool tc_supported(const Ctx& ctx, const ScoreArgs& a) {
   // tensor-map limits: strides below 2^40 bytes, multiples of 16 bytes (checked by the caller)
   if (a.k_stride_token * 2 >= (1ll << 40) || a.k_stride_head * 2 >= (1ll << 40)) return false;
   if (ctx.cfg.n_kv_heads > 1 && a.k_stride_head == 0) return false;
+  const int rows_pg = (ctx.cfg.n_q_heads / ctx.cfg.n_kv_heads) * w;
+  if (ctx.cfg.n_kv_heads * ((rows_pg + kRowBlock - 1) / kRowBlock) > kQueueUnits) return false;   // work-queue slots
   return true;
 }
 
@@ -966,26 +1037,44 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.q_rows = ctx.cfg.n_q_heads * ctx.cfg.window;
   p.rows_all = (long long)a.batch * ctx.rows_pad;
   // The CTAs of the grid (about one per SM) are shared out over the sequences in proportion to
-  // their lengths; every (KV group, row block) unit of a sequence gets the same number of key
-  // segments, at least one, at most one per pair of key tiles.
-  const int units = ctx.cfg.n_kv_heads * p.n_rb;
+  // their lengths, and inside a KV group over its row blocks in proportion to their cost: a last
+  // block that holds a single 128-row half costs half a full block per key tile in pass 1 and
+  // between a half and three quarters in pass 2 (fewer warps share its exponentials), 0.65 over
+  // both.  Every unit gets at least one key segment and at most one per pair of key tiles.
+  const int halves_last = (p.rows_pg - (p.n_rb - 1) * kRowBlock + 127) / 128;       // 1 or 2
+  const double weight_last = halves_last == 2 ? 1.0 : 0.65;
+  const double group_weight = (double)(p.n_rb - 1) + weight_last;
   int grid = 0, max_segs = 0;
   for (int b = 0; b < a.batch; ++b) {
     const int key0 = a.cu_seqlens ? a.cu_seqlens[b] : 0;
     const int n_b = a.cu_seqlens ? a.cu_seqlens[b + 1] - key0 : a.n_keys;
     const int n_pairs = ((n_b + kKeyTile - 1) / kKeyTile + 1) / 2;
-    int segs = (int)((double)ctx.sm_count * n_b / ((double)a.total_keys * units));
-    if (segs < 1) segs = 1;
-    if (segs > n_pairs) segs = n_pairs;
-    if (segs > kMaxParts) segs = kMaxParts;         // pass 1 leaves one partial statistic per segment
-    p.seq[b] = SeqDesc{key0, n_b, grid, segs};
-    grid += units * segs;
+    const double per_group = (double)ctx.sm_count * n_b / ((double)a.total_keys * ctx.cfg.n_kv_heads);
+    auto clamp_segs = [&](int v) { return v < 1 ? 1 : (v > n_pairs ? n_pairs : (v > kMaxParts ? kMaxParts : v)); };
+    // pass 1 leaves one partial statistic per segment, hence the bound kMaxParts
+    const int segs = clamp_segs((int)(per_group / group_weight));
+    const int segs_last = p.n_rb == 1 ? segs : clamp_segs((int)(weight_last * segs + 0.5));
+    p.seq[b] = SeqDesc{key0, n_b, grid, segs, segs_last};
+    grid += ctx.cfg.n_kv_heads * ((p.n_rb - 1) * segs + segs_last);
     if (segs > max_segs) max_segs = segs;
+    if (segs_last > max_segs) max_segs = segs_last;
   }
   p.c2 = a.scale * kLog2e;
   // the fold needs a finite lse / c2 (a zero scale keeps the plain form)
   p.fold = (SKV_FOLD != 0) && pass == 2 && fabsf(p.c2) > 1e-20f ? 1 : 0;
   p.inputs_ready = a.inputs_ready ? 1 : 0;
+  // tickets of pass 2: every unit's counter advances, per launch, by its tiles plus one failed draw
+  // per CTA.  A plain call has equal units, so one base serves them all; a batch starts from
+  // zeroed counters.
+  p.queue = ctx.ws.queue;
+  p.queue_base = ctx.queue_base;
+  p.queue_base_last = ctx.queue_base_last;
+  unsigned long long advance = 0, advance_last = 0;
+  if (!a.cu_seqlens && pass == 2) {
+    const unsigned long long n_tiles = (unsigned long long)((a.n_keys + kKeyTile - 1) / kKeyTile);
+    advance = n_tiles + (unsigned long long)p.seq[0].segs;
+    advance_last = n_tiles + (unsigned long long)p.seq[0].segs_last;
+  }
   p.inv_c2 = p.fold ? 1.0f / p.c2 : 0.f;
   p.row_part = ctx.ws.row_part;
   p.row_ent = ctx.ws.row_ent;
@@ -994,8 +1083,14 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.status = ctx.ws.status;
   *parts_out = max_segs;
   const int d = ctx.cfg.head_dim, w = ctx.cfg.window;
-  if (d == 128) return pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);
-  return pass == 1 ? launch_w<64, 1>(w, mq, mk, p, grid, st) : launch_w<64, 2>(w, mq, mk, p, grid, st);
+  cudaError_t e;
+  if (d == 128) e = pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);
+  else e = pass == 1 ? launch_w<64, 1>(w, mq, mk, p, grid, st) : launch_w<64, 2>(w, mq, mk, p, grid, st);
+  if (e == cudaSuccess) {                            // the counters move only if the kernel runs
+    ctx.queue_base += advance;
+    ctx.queue_base_last += advance_last;
+  }
+  return e;
 }
 
 }  // namespace skv
