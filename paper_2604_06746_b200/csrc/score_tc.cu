@@ -602,7 +602,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       const int row_lo = quarter * 32 + lane;
       const int i_win = row_lo % p.window;          // window row of this thread's rows (the window divides 128)
       const int t_pos = n_keys - p.window + i_win;                     // their position: they see keys <= t_pos
-      const int first_tail_pair = (n_keys - p.window + 1) / (2 * kKeyTile);
+      const int last_open_key = n_keys - p.window;               // the last key every window row sees
       // Z += 2^(x - ref), U += 2^(x - ref) (x - ref) over one chunk whose keys are all visible;
       // of every 8 elements the first kPoly1 are exponentiated on the FMA pipe
       auto accumulate = [&](RowStat& r) {
@@ -673,18 +673,21 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
             const int item = acc_full(u);                 // the same pair for both row halves
             if (item < 0) { live = false; continue; }
             const int jb = item * (2 * kKeyTile) + sub * 64;
-            const bool plain = item < first_tail_pair;
+            // a 32-key chunk takes the plain path when every window row sees all of its keys; of
+            // the sequence's last pair only the chunks that hold window keys (or lie beyond the
+            // sequence) take the masked one
+            const bool plain0 = jb + 31 <= last_open_key, plain1 = jb + 63 <= last_open_key;
             const bool warp_active = (hf * 128 + quarter * 32) < rows_here;
             const uint32_t taddr = tmem + lane_base + (uint32_t)((u % kAccStages) * 256 + sub * 64);
             if (warp_active) {
               tmem_ld32(taddr, v);
               tmem_ld_wait(v);
-              chunk(st[hf], jb, plain && t > 0);          // the first pair gives the rows their reference
+              chunk(st[hf], jb, plain0 && t > 0);         // the first pair gives the rows their reference
               tmem_ld32(taddr + 32, v);
               tmem_ld_wait(v);
             }
             acc_release(u);
-            if (warp_active) chunk(st[hf], jb + 32, plain);
+            if (warp_active) chunk(st[hf], jb + 32, plain1);
             ++u;
           }
         }
