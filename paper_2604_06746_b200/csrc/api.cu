@@ -49,7 +49,7 @@ Workspace carve_workspace(const structkv_config& cfg, void* base) {
   w.row_ent = (float*)take(rows_pad * sizeof(float));
   w.cols = (float*)take((size_t)cfg.n_q_heads * n_pad * sizeof(float));
   w.head_part = (float*)take((size_t)kMaxStatLayers * cfg.n_q_heads * 4 * sizeof(float));
-  w.queue = (unsigned long long*)take((size_t)kQueueUnits * sizeof(unsigned long long));
+  w.queue = (unsigned long long*)take((size_t)kMaxBatch * kQueueUnits * sizeof(unsigned long long));
   w.bytes = off;
   return w;
 }
@@ -100,7 +100,7 @@ structkv_status structkv_create(structkv_ctx** ctx_out, const structkv_config* c
   if (cudaGetDevice(&c.device) != cudaSuccess ||
       cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess ||
       cudaMemset(c.ws.status, 0, 256) != cudaSuccess ||
-      cudaMemset(c.ws.queue, 0, (size_t)kQueueUnits * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMemset(c.ws.queue, 0, (size_t)kMaxBatch * kQueueUnits * sizeof(unsigned long long)) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess) {
     delete ctx;
     return STRUCTKV_ERR_CUDA;
@@ -168,7 +168,7 @@ structkv_status structkv_score_layer(structkv_ctx* ctx, const void* q_window, co
 
 // ---- batches of prompts of different lengths (packed along the token axis) ------------------
 namespace skv {
-struct BatchWs { float4* row_part; float* row_ent; float* cols; float* head_part; unsigned long long* queue; size_t bytes; };
+struct BatchWs { float4* row_part; float* row_ent; float* cols; float* head_part; size_t bytes; };
 static BatchWs carve_batch(const structkv_config& cfg, int max_batch, long long max_total, void* base) {
   BatchWs w{};
   char* p = (char*)base;
@@ -184,7 +184,6 @@ static BatchWs carve_batch(const structkv_config& cfg, int max_batch, long long 
   w.row_ent = (float*)take(rows_all * sizeof(float));
   w.cols = (float*)take((size_t)cfg.n_q_heads * t_pad * sizeof(float));
   w.head_part = (float*)take((size_t)max_batch * cfg.n_q_heads * 4 * sizeof(float));
-  w.queue = (unsigned long long*)take((size_t)max_batch * kQueueUnits * sizeof(unsigned long long));
   w.bytes = off;
   return w;
 }
@@ -229,11 +228,7 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   view.ws.row_ent = bw.row_ent;
   view.ws.cols = bw.cols;
   view.ws.head_part = bw.head_part;
-  // the batch's own ticket counters start from zero in every call (the workspace is the caller's)
-  view.ws.queue = bw.queue;
-  view.queue_base = view.queue_base_last = 0;
-  if (cudaMemsetAsync(bw.queue, 0, (size_t)batch * kQueueUnits * sizeof(unsigned long long), st) != cudaSuccess)
-    return STRUCTKV_ERR_CUDA;
+  // the ticket counters stay the context's own (its workspace is known to be initialised)
   ScoreArgs a;
   a.q = q_window; a.k = k;
   a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
@@ -247,6 +242,7 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   int parts = 0;
   if (launch_score_tc(view, a, &parts, 1, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
   if (launch_score_tc(view, a, &parts, 2, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
+  std::memcpy(c.queue_base, view.queue_base, sizeof(c.queue_base));   // the launches advanced the view's copy
   // per sequence: S = sum over heads, C <- lambda C + S, and the sequence's metric triple
   for (int b = 0; b < batch; ++b) {
     const int key0 = cu_seqlens[b], n_b = cu_seqlens[b + 1] - key0;
@@ -449,10 +445,10 @@ structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream) {
     // a scorer launch that gave up may have left its ticket counters short of what the host
     // expects: start them over together with the status word
     if (cudaMemsetAsync(ctx->c.ws.status, 0, sizeof(int), st) != cudaSuccess ||
-        cudaMemsetAsync(ctx->c.ws.queue, 0, (size_t)kQueueUnits * sizeof(unsigned long long), st) != cudaSuccess ||
+        cudaMemsetAsync(ctx->c.ws.queue, 0, (size_t)kMaxBatch * kQueueUnits * sizeof(unsigned long long), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
       return STRUCTKV_ERR_CUDA;
-    ctx->c.queue_base = ctx->c.queue_base_last = 0;
+    std::memset(ctx->c.queue_base, 0, sizeof(ctx->c.queue_base));
   }
   if (word < 0 || word > (int)STRUCTKV_ERR_TIMEOUT) return STRUCTKV_ERR_CUDA;
   return (structkv_status)word;
@@ -530,7 +526,7 @@ extern "C" structkv_status structkv_score_layer_static(
   // The scratch keeps the previous call's contents; the status word must start from zero.
   if (cudaMemsetAsync(c.ws.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return STRUCTKV_ERR_CUDA;
   // the per-call context starts its ticket counters from zero as well
-  if (cudaMemsetAsync(c.ws.queue, 0, (size_t)kQueueUnits * sizeof(unsigned long long), (cudaStream_t)stream) !=
+  if (cudaMemsetAsync(c.ws.queue, 0, (size_t)kMaxBatch * kQueueUnits * sizeof(unsigned long long), (cudaStream_t)stream) !=
       cudaSuccess)
     return STRUCTKV_ERR_CUDA;
   return structkv_score_layer(&tmp, q_window, k, k_stride_head, k_stride_token, n_keys, scale, lambda,

@@ -27,9 +27,10 @@ struct Workspace {
   float* row_ent;       // [rows_pad] entropy of each score row (nats)
   float* cols;          // [H][n_pad] pooled per-head attention when the caller passes none
   float* head_part;     // [kMaxStatLayers][H][4] per-(layer, head) {sum of squared deviations from 1/n, top-k mass}
-  // [kQueueUnits] ticket counters of the tensor-core scorer's second pass, one per (KV group,
-  // row block); zero when the context is created, never reset: every launch advances them by a
-  // known amount (queue_base in Ctx follows)
+  // [kMaxBatch][kQueueUnits] ticket counters of the tensor-core scorer's second pass, one per
+  // (sequence slot of a call, KV group, row block); zero when the context is created, never
+  // reset: every launch advances the counters of the slots it uses by a known amount
+  // (queue_base in Ctx follows)
   unsigned long long* queue;
   size_t bytes;
 };
@@ -43,8 +44,9 @@ struct Ctx {
   int rows_pad;         // rows per KV group padded to kRowBlock, times H_kv
   int n_pad;            // max_seq rounded up to kKeyTile
   void* tc;             // tensor-core scorer state (tensor maps), owned by score_tc.cu
-  unsigned long long queue_base = 0;        // first ticket of the next launch of the scorer's second pass (units on full row blocks)
-  unsigned long long queue_base_last = 0;   // the same for the units on a KV group's last row block
+  // first ticket of the next launch of the scorer's second pass, per sequence slot: [0] for the
+  // units on full row blocks, [1] for the units on a KV group's last row block
+  unsigned long long queue_base[kMaxBatch][2] = {};
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

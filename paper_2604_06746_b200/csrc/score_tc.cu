@@ -43,7 +43,10 @@ constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 
 // row block of a KV group is worked on by `segs` CTAs and the group's last row block by
 // `segs_last` (fewer when it holds only one 128-row half), so a group takes
 // (n_rb - 1) * segs + segs_last consecutive CTAs from cta0 on.  A plain call is a batch of one.
-struct SeqDesc { int key0, n_keys, cta0, segs, segs_last; };
+struct SeqDesc {
+  int key0, n_keys, cta0, segs, segs_last;
+  unsigned long long ticket0, ticket0_last;   // pass 2: this launch's first ticket on full row blocks / on the last one
+};
 
 struct TcParams {
   int window, group, rows_pg, rows_pg_pad, rows_pad, n_rb;
@@ -57,9 +60,8 @@ struct TcParams {
   int inputs_ready;                    // pass 1: Q and K are complete and visible, no kernel in flight writes them
   // Work queue of pass 2: one ticket counter per (sequence, KV group, row block); a CTA draws
   // key tiles of its unit from it until the unit has none left.  The counters only ever grow;
-  // a launch's tickets start at queue_base.
+  // a launch's tickets start at the sequence's ticket0.
   unsigned long long* queue;
-  unsigned long long queue_base, queue_base_last;   // units on full row blocks / on a group's last row block
   float4* row_part;                    // pass 1 out, pass 2 in: [segs][n_seq][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): [n_seq][rows_pad] entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride], sequence b at column key0_b
@@ -380,7 +382,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   const int t_lo = (int)((long long)seg * n_items / segs);          // pass 1: first pair of this CTA
   const int n_static = (int)((long long)(seg + 1) * n_items / segs) - t_lo;
   const int units_per_seq = p.n_rb * (p.rows_pad / p.rows_pg_pad);
-  unsigned long long* const ticket = p.queue + (size_t)sq * units_per_seq + unit;
+  unsigned long long* const ticket = p.queue + (size_t)sq * kQueueUnits + unit;
   int* item_s = reinterpret_cast<int*>(sm + L::kBarOff + 8 * kBarCount + 32);      // producer -> MMA issuer, per K slot
   volatile int* unit_item = reinterpret_cast<volatile int*>(sm + L::kBarOff + 8 * kBarCount + 48);   // MMA issuer -> compute warps, per accumulator stage
   const int rows_here = min(kRowBlock, p.rows_pg - rb * kRowBlock);     // valid score rows in this block
@@ -440,7 +442,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         if (PASS == 1) {
           item = it < n_static ? t_lo + it : -1;
         } else {
-          const long long idx = (long long)(tk - (rb == p.n_rb - 1 ? p.queue_base_last : p.queue_base));
+          const long long idx = (long long)(tk - (rb == p.n_rb - 1 ? p.seq[sq].ticket0_last : p.seq[sq].ticket0));
           item = idx < (long long)n_items ? n_items - 1 - (int)idx : -1;
           if (item >= 0) tk = atomicAdd(ticket, 1ull);     // the next ticket travels while this tile is loaded
         }
@@ -1057,7 +1059,7 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
     // pass 1 leaves one partial statistic per segment, hence the bound kMaxParts
     const int segs = clamp_segs((int)(per_group / group_weight));
     const int segs_last = p.n_rb == 1 ? segs : clamp_segs((int)(weight_last * segs + 0.5));
-    p.seq[b] = SeqDesc{key0, n_b, grid, segs, segs_last};
+    p.seq[b] = SeqDesc{key0, n_b, grid, segs, segs_last, ctx.queue_base[b][0], ctx.queue_base[b][1]};
     grid += ctx.cfg.n_kv_heads * ((p.n_rb - 1) * segs + segs_last);
     if (segs > max_segs) max_segs = segs;
     if (segs_last > max_segs) max_segs = segs_last;
@@ -1067,17 +1069,8 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   p.fold = (SKV_FOLD != 0) && pass == 2 && fabsf(p.c2) > 1e-20f ? 1 : 0;
   p.inputs_ready = a.inputs_ready ? 1 : 0;
   // tickets of pass 2: every unit's counter advances, per launch, by its tiles plus one failed draw
-  // per CTA.  A plain call has equal units, so one base serves them all; a batch starts from
-  // zeroed counters.
+  // per CTA of the unit
   p.queue = ctx.ws.queue;
-  p.queue_base = ctx.queue_base;
-  p.queue_base_last = ctx.queue_base_last;
-  unsigned long long advance = 0, advance_last = 0;
-  if (!a.cu_seqlens && pass == 2) {
-    const unsigned long long n_tiles = (unsigned long long)((a.n_keys + kKeyTile - 1) / kKeyTile);
-    advance = n_tiles + (unsigned long long)p.seq[0].segs;
-    advance_last = n_tiles + (unsigned long long)p.seq[0].segs_last;
-  }
   p.inv_c2 = p.fold ? 1.0f / p.c2 : 0.f;
   p.row_part = ctx.ws.row_part;
   p.row_ent = ctx.ws.row_ent;
@@ -1089,10 +1082,12 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   cudaError_t e;
   if (d == 128) e = pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);
   else e = pass == 1 ? launch_w<64, 1>(w, mq, mk, p, grid, st) : launch_w<64, 2>(w, mq, mk, p, grid, st);
-  if (e == cudaSuccess) {                            // the counters move only if the kernel runs
-    ctx.queue_base += advance;
-    ctx.queue_base_last += advance_last;
-  }
+  if (e == cudaSuccess && pass == 2)                 // the counters move only if the kernel runs
+    for (int b = 0; b < a.batch; ++b) {
+      const unsigned long long n_tiles = (unsigned long long)((p.seq[b].n_keys + kKeyTile - 1) / kKeyTile);
+      ctx.queue_base[b][0] += n_tiles + (unsigned long long)p.seq[b].segs;
+      ctx.queue_base[b][1] += n_tiles + (unsigned long long)p.seq[b].segs_last;
+    }
   return e;
 }
 
