@@ -242,7 +242,7 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   int parts = 0;
   if (launch_score_tc(view, a, &parts, 1, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
   if (launch_score_tc(view, a, &parts, 2, st) != cudaSuccess) return STRUCTKV_ERR_CUDA;
-  std::memcpy(c.queue_base, view.queue_base, sizeof(c.queue_base));   // the launches advanced the view's copy
+  std::memcpy(c.queue_period, view.queue_period, sizeof(c.queue_period));   // the launches updated the view's copy
   // per sequence: S = sum over heads, C <- lambda C + S, and the sequence's metric triple
   for (int b = 0; b < batch; ++b) {
     const int key0 = cu_seqlens[b], n_b = cu_seqlens[b + 1] - key0;
@@ -448,7 +448,7 @@ structkv_status structkv_poll_device_status(structkv_ctx* ctx, void* stream) {
         cudaMemsetAsync(ctx->c.ws.queue, 0, (size_t)kMaxBatch * kQueueUnits * sizeof(unsigned long long), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
       return STRUCTKV_ERR_CUDA;
-    std::memset(ctx->c.queue_base, 0, sizeof(ctx->c.queue_base));
+    std::memset(ctx->c.queue_period, 0, sizeof(ctx->c.queue_period));
   }
   if (word < 0 || word > (int)STRUCTKV_ERR_TIMEOUT) return STRUCTKV_ERR_CUDA;
   return (structkv_status)word;

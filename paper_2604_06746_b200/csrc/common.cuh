@@ -28,9 +28,11 @@ struct Workspace {
   float* cols;          // [H][n_pad] pooled per-head attention when the caller passes none
   float* head_part;     // [kMaxStatLayers][H][4] per-(layer, head) {sum of squared deviations from 1/n, top-k mass}
   // [kMaxBatch][kQueueUnits] ticket counters of the tensor-core scorer's second pass, one per
-  // (sequence slot of a call, KV group, row block); zero when the context is created, never
-  // reset: every launch advances the counters of the slots it uses by a known amount
-  // (queue_base in Ctx follows)
+  // (sequence slot of a call, KV group, row block); zero when the context is created.  A launch
+  // draws exactly T = tiles + CTAs-of-the-unit tickets from a unit's counter and reads a ticket
+  // modulo T, so launches of one shape follow each other with no reset and no per-launch host
+  // state (a captured launch can be replayed); the host zeroes a slot only when its T changes
+  // (queue_period in Ctx)
   unsigned long long* queue;
   size_t bytes;
 };
@@ -44,9 +46,9 @@ struct Ctx {
   int rows_pad;         // rows per KV group padded to kRowBlock, times H_kv
   int n_pad;            // max_seq rounded up to kKeyTile
   void* tc;             // tensor-core scorer state (tensor maps), owned by score_tc.cu
-  // first ticket of the next launch of the scorer's second pass, per sequence slot: [0] for the
-  // units on full row blocks, [1] for the units on a KV group's last row block
-  unsigned long long queue_base[kMaxBatch][2] = {};
+  // tickets per launch (T) the counters of a sequence slot were last used with: [0] for the units
+  // on full row blocks, [1] for the units on a KV group's last row block; 0 = counters are zero
+  unsigned int queue_period[kMaxBatch][2] = {};
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -45,7 +45,7 @@ constexpr float kMasked = -1.0e30f;    // stands for -inf: 2^x flushes to 0 and 
 // (n_rb - 1) * segs + segs_last consecutive CTAs from cta0 on.  A plain call is a batch of one.
 struct SeqDesc {
   int key0, n_keys, cta0, segs, segs_last;
-  unsigned long long ticket0, ticket0_last;   // pass 2: this launch's first ticket on full row blocks / on the last one
+  unsigned int period, period_last;   // pass 2: tickets one launch draws from a unit's counter (tiles + CTAs of the unit)
 };
 
 struct TcParams {
@@ -60,7 +60,7 @@ struct TcParams {
   int inputs_ready;                    // pass 1: Q and K are complete and visible, no kernel in flight writes them
   // Work queue of pass 2: one ticket counter per (sequence, KV group, row block); a CTA draws
   // key tiles of its unit from it until the unit has none left.  The counters only ever grow;
-  // a launch's tickets start at the sequence's ticket0.
+  // a ticket is read modulo the number of tickets one launch draws (SeqDesc::period).
   unsigned long long* queue;
   float4* row_part;                    // pass 1 out, pass 2 in: [segs][n_seq][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): [n_seq][rows_pad] entropy of each score row, nats
@@ -442,8 +442,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
         if (PASS == 1) {
           item = it < n_static ? t_lo + it : -1;
         } else {
-          const long long idx = (long long)(tk - (rb == p.n_rb - 1 ? p.seq[sq].ticket0_last : p.seq[sq].ticket0));
-          item = idx < (long long)n_items ? n_items - 1 - (int)idx : -1;
+          const int idx = (int)(tk % (unsigned long long)(rb == p.n_rb - 1 ? p.seq[sq].period_last : p.seq[sq].period));
+          item = idx < n_items ? n_items - 1 - idx : -1;
           if (item >= 0) tk = atomicAdd(ticket, 1ull);     // the next ticket travels while this tile is loaded
         }
         const int s0 = (kPerItem * it) % kStages;
@@ -1059,7 +1059,8 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
     // pass 1 leaves one partial statistic per segment, hence the bound kMaxParts
     const int segs = clamp_segs((int)(per_group / group_weight));
     const int segs_last = p.n_rb == 1 ? segs : clamp_segs((int)(weight_last * segs + 0.5));
-    p.seq[b] = SeqDesc{key0, n_b, grid, segs, segs_last, ctx.queue_base[b][0], ctx.queue_base[b][1]};
+    const unsigned int n_tiles_b = (unsigned int)((n_b + kKeyTile - 1) / kKeyTile);
+    p.seq[b] = SeqDesc{key0, n_b, grid, segs, segs_last, n_tiles_b + (unsigned int)segs, n_tiles_b + (unsigned int)segs_last};
     grid += ctx.cfg.n_kv_heads * ((p.n_rb - 1) * segs + segs_last);
     if (segs > max_segs) max_segs = segs;
     if (segs_last > max_segs) max_segs = segs_last;
@@ -1068,9 +1069,22 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   // the fold needs a finite lse / c2 (a zero scale keeps the plain form)
   p.fold = (SKV_FOLD != 0) && pass == 2 && fabsf(p.c2) > 1e-20f ? 1 : 0;
   p.inputs_ready = a.inputs_ready ? 1 : 0;
-  // tickets of pass 2: every unit's counter advances, per launch, by its tiles plus one failed draw
-  // per CTA of the unit
+  // tickets of pass 2: a unit's counter advances, per launch, by its tiles plus one failed draw per
+  // CTA of the unit, and tickets are read modulo that number.  A slot whose number changes (another
+  // sequence length) starts again from zero; this is settled before pass 1, so that nothing comes
+  // between the two passes.
   p.queue = ctx.ws.queue;
+  if (pass == 1)
+    for (int b = 0; b < a.batch; ++b) {
+      const unsigned int want[2] = {p.seq[b].period, p.seq[b].period_last};
+      const bool stale = (ctx.queue_period[b][0] != 0 && ctx.queue_period[b][0] != want[0]) ||
+                         (ctx.queue_period[b][1] != 0 && ctx.queue_period[b][1] != want[1]);
+      if (stale && cudaMemsetAsync(ctx.ws.queue + (size_t)b * kQueueUnits, 0,
+                                   (size_t)kQueueUnits * sizeof(unsigned long long), st) != cudaSuccess)
+        return cudaErrorUnknown;
+      ctx.queue_period[b][0] = want[0];
+      ctx.queue_period[b][1] = want[1];
+    }
   p.inv_c2 = p.fold ? 1.0f / p.c2 : 0.f;
   p.row_part = ctx.ws.row_part;
   p.row_ent = ctx.ws.row_ent;
@@ -1082,12 +1096,6 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   cudaError_t e;
   if (d == 128) e = pass == 1 ? launch_w<128, 1>(w, mq, mk, p, grid, st) : launch_w<128, 2>(w, mq, mk, p, grid, st);
   else e = pass == 1 ? launch_w<64, 1>(w, mq, mk, p, grid, st) : launch_w<64, 2>(w, mq, mk, p, grid, st);
-  if (e == cudaSuccess && pass == 2)                 // the counters move only if the kernel runs
-    for (int b = 0; b < a.batch; ++b) {
-      const unsigned long long n_tiles = (unsigned long long)((p.seq[b].n_keys + kKeyTile - 1) / kKeyTile);
-      ctx.queue_base[b][0] += n_tiles + (unsigned long long)p.seq[b].segs;
-      ctx.queue_base[b][1] += n_tiles + (unsigned long long)p.seq[b].segs_last;
-    }
   return e;
 }
 

@@ -330,3 +330,32 @@ def test_batched_head_statistics_on_unaligned_vectors(mods, cuda_device):
         P.assert_metric_close(got[l, 1], rho, f"sparsity of layer {l}")
         P.assert_metric_close(got[l, 2], var, f"variance of layer {l}")
     ctx.close()
+
+
+def test_a_captured_layer_can_be_replayed(mods, cuda_device):
+    """structkv_score_layer keeps no per-launch state on the host (the second pass reads its work
+    tickets modulo the number one launch draws), so a call captured into a CUDA graph gives the
+    eager call's bits on every replay, also with eager calls of the same shape in between."""
+    binding, _ = mods
+    wl = synth.WORKLOADS["llama32k"].scaled(6000 + 19, n_layers=1, n_hubs=4, budgets=(256,))
+    t = synth.make_layer(wl, synth.plan(wl), 0, device="cpu", with_v=False)
+    q, k = t["q_win"].to(cuda_device), t["k"].to(cuda_device)
+    ctx = binding.Context(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window, wl.seq, torch.bfloat16, cuda_device)
+    s_e, s_g = (torch.zeros(wl.seq, device=cuda_device) for _ in range(2))
+    m_e, m_g = (torch.zeros(3, device=cuda_device) for _ in range(2))
+    for _ in range(2):
+        ctx.score_layer(q, k, t["scale"], s_e, m_e)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.score_layer(q, k, t["scale"], s_g, m_g)
+    for i in range(4):
+        s_g.zero_(); m_g.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(s_g, s_e) and torch.equal(m_g, m_e), f"replay {i}"
+        if i == 1:
+            ctx.score_layer(q, k, t["scale"], s_e, m_e)       # an eager call between replays
+            torch.cuda.synchronize()
+    assert ctx.poll_device_status() == binding.OK
+    ctx.close()
