@@ -192,8 +192,7 @@ class Resident:
         pf, layers = self.pf, self.layers
         e = [ev() for _ in range(4)] if timed else None
         if timed: e[0].record()
-        for l, t in enumerate(layers):
-            pf.score(l, t["q_win"], t["k"], t["scale"])
+        pf.score_all(layers)                   # all layers resident: one call, passes of neighbouring layers interleaved
         pf.finish_scores(len(layers))          # Eq. 5-6 of all layers (batched): part of the scoring phase
         if timed: e[1].record()
         pf.detect_and_select(len(layers))
@@ -377,12 +376,15 @@ def compaction_figures(wl, kv_budget, compact_ms_per_step, peaks):
 
 def launches_per_step(wl, flags):
     from paper_2604_06746_b200 import binding
-    # per layer: scorer pass 1, pass 2, column reduce + metrics (the CUDA-core scorer adds a row
+    # layer by layer: scorer pass 1, pass 2, column reduce + metrics (the CUDA-core scorer adds a row
     # finalisation); per step: batched head statistics (2), accumulate, 2 selections, one K/V gather
     # over all layers, hidden states, positions
-    per_layer = 3 if wl.dtype == "bf16" else 4
     stats = 0 if (flags & binding.FLAG_NO_HEAD_STATS) else 2
-    return wl.n_layers * per_layer + stats + 1 + 2 + 1 + 2
+    if wl.dtype == "bf16" and not (flags & (binding.FLAG_NO_HEAD_STATS | binding.FLAG_FORCE_SIMT)):
+        scoring = 2 * wl.n_layers + 1          # one structkv_score_layers call: two passes per layer, one reduce over heads
+    else:
+        scoring = wl.n_layers * (3 if wl.dtype == "bf16" else 4)
+    return scoring + stats + 1 + 2 + 1 + 2
 
 
 # ------------------------------------------------------------------------------------------------

@@ -169,6 +169,40 @@ structkv_status structkv_select_batch(structkv_ctx* ctx, const float* scores, co
                                       long long idx_stride, void* stream);
 
 /*
+ * Algorithm 1 lines 3-6 (Eq. 1-4) for SEVERAL layers whose window queries and keys are all
+ * resident (a prompt whose KV cache already exists, or a prefill that ran ahead of the scoring).
+ * Per layer the results are the very bits structkv_score_layer gives with
+ * STRUCTKV_FLAG_NO_HEAD_STATS: S^(l), the pooled per-head attention, the layer's entropy; C is
+ * carried through all layers (C <- lambda*C + S^(l), l ascending).  What differs is the order of
+ * the work: the first scorer pass of layer l+1 is enqueued between the two passes of layer l, and
+ * the second pass of layer l waits for a completion counter of its own first pass instead of for
+ * the kernel enqueued before it, so no SM idles while the slowest CTA of a pass finishes; the
+ * sums over heads of all layers are taken by one launch at the end.
+ *
+ *   q_windows, ks  HOST arrays [n_layers] of device pointers, laid out as for structkv_score_layer
+ *                 (one stride pair serves all layers); every tensor must be complete and visible
+ *                 before the call is enqueued (as with STRUCTKV_FLAG_INPUTS_READY).
+ *   scales        HOST array [n_layers].
+ *   s_out         device, fp32: S^(l) at s_out + l*s_layer_stride, s_layer_stride >= n_keys.
+ *   c_inout       device, [n_keys] fp32 or NULL.
+ *   head_cols_out device, fp32, required: layer l's [H, n_keys] slab at
+ *                 head_cols_out + l*head_cols_layer_stride (feed it to structkv_head_stats).
+ *   metrics_out   device, [n_layers, 3] fp32: [l][0] = entropy, [l][1..2] = NaN.
+ *   layers_workspace  device, 256-byte aligned, at least structkv_layers_workspace_bytes(cfg, n_layers)
+ *                 bytes, caller-owned.
+ * Shapes the tensor-core scorer does not take are scored layer after layer (same results).
+ * Errors: INVALID_ARG, WORKSPACE, CUDA.  Asynchronous on `stream`.
+ */
+size_t structkv_layers_workspace_bytes(const structkv_config* cfg, int max_layers);
+structkv_status structkv_score_layers(structkv_ctx* ctx, int n_layers, const void* const* q_windows,
+                                      const void* const* ks, long long k_stride_head,
+                                      long long k_stride_token, int n_keys, const float* scales, float lambda,
+                                      float* s_out, long long s_layer_stride, float* c_inout,
+                                      float* head_cols_out, long long head_cols_layer_stride,
+                                      float* metrics_out, void* layers_workspace,
+                                      size_t layers_workspace_bytes, void* stream);
+
+/*
  * Eq. 5 and Eq. 6 (Section 3.3) for several layers at once, from the pooled per-head attention
  * that structkv_score_layer wrote to head_cols_out.  A caller that scores many layers passes
  * STRUCTKV_FLAG_NO_HEAD_STATS and a distinct head_cols_out slab per layer, then makes ONE call

@@ -58,6 +58,11 @@ lib.structkv_batch_workspace_bytes.argtypes = [ctypes.POINTER(Config), _i, _ll]
 lib.structkv_score_layer_batch.restype = _i
 lib.structkv_score_layer_batch.argtypes = [_vp, _vp, _vp, _ll, _ll, ctypes.POINTER(_i), _i, _f, _f, _vp, _vp, _vp,
                                            _vp, _u, _vp, ctypes.c_size_t, _vp]
+lib.structkv_layers_workspace_bytes.restype = ctypes.c_size_t
+lib.structkv_layers_workspace_bytes.argtypes = [ctypes.POINTER(Config), _i]
+lib.structkv_score_layers.restype = _i
+lib.structkv_score_layers.argtypes = [_vp, _i, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ll, _ll, _i,
+                                      ctypes.POINTER(_f), _f, _vp, _ll, _vp, _vp, _ll, _vp, _vp, ctypes.c_size_t, _vp]
 lib.structkv_select_batch.restype = _i
 lib.structkv_select_batch.argtypes = [_vp, _vp, ctypes.POINTER(_i), ctypes.POINTER(_i), _i, _i, _vp, _ll, _vp]
 lib.structkv_head_stats.restype = _i
@@ -197,6 +202,34 @@ class Context:
                                               _ptr(head_cols_out), metrics_out.data_ptr(), flags,
                                               workspace.data_ptr(), workspace.numel(), _stream(stream)),
                "structkv_score_layer_batch")
+
+    def score_layers(self, q_windows: Sequence[torch.Tensor], ks: Sequence[torch.Tensor], scales: Sequence[float],
+                     s_out: torch.Tensor, metrics_out: torch.Tensor, head_cols_out: torch.Tensor,
+                     workspace: torch.Tensor, c_inout: Optional[torch.Tensor] = None, lam: float = 0.9,
+                     stream: Optional[torch.cuda.Stream] = None) -> None:
+        """structkv_score_layers: layer ``l`` takes ``q_windows[l] [H, w, d]`` and ``ks[l] [H_kv, N, d]`` (all
+        with the strides of ``ks[0]``); ``s_out [L, N]``, ``head_cols_out [L, H, N]``, ``metrics_out [L, 3]``."""
+        L = len(q_windows)
+        k0 = ks[0]
+        assert len(ks) == L and len(scales) == L and L >= 1
+        assert all(q.is_contiguous() for q in q_windows)
+        assert all(k.shape == k0.shape and k.stride() == k0.stride() and k.stride(2) == 1 for k in ks)
+        n = k0.shape[1]
+        assert s_out.shape == (L, n) and s_out.stride(1) == 1 and metrics_out.is_contiguous()
+        assert metrics_out.shape == (L, 3) and head_cols_out.shape[0] == L and head_cols_out[0].is_contiguous()
+        qp = (_vp * L)(*[q.data_ptr() for q in q_windows])
+        kp = (_vp * L)(*[k.data_ptr() for k in ks])
+        sc = (_f * L)(*scales)
+        _check(lib.structkv_score_layers(self._h, L, qp, kp, k0.stride(0), k0.stride(1), n, sc, lam,
+                                         s_out.data_ptr(), s_out.stride(0), _ptr(c_inout), head_cols_out.data_ptr(),
+                                         head_cols_out.stride(0), metrics_out.data_ptr(), workspace.data_ptr(),
+                                         workspace.numel(), _stream(stream)), "structkv_score_layers")
+
+    def layers_workspace(self, max_layers: int) -> torch.Tensor:
+        n = lib.structkv_layers_workspace_bytes(ctypes.byref(self.cfg), max_layers)
+        if n == 0:
+            raise StructKVError(ERR_INVALID_ARG, "structkv_layers_workspace_bytes")
+        return torch.empty(n, dtype=torch.uint8, device=self.device)
 
     def batch_workspace(self, max_batch: int, max_total_tokens: int) -> torch.Tensor:
         n = lib.structkv_batch_workspace_bytes(ctypes.byref(self.cfg), max_batch, max_total_tokens)

@@ -257,6 +257,118 @@ structkv_status structkv_score_layer_batch(structkv_ctx* ctx, const void* q_wind
   return STRUCTKV_OK;
 }
 
+// ---- several resident layers in one call, the passes of neighbouring layers interleaved ---------
+namespace skv {
+struct LayersWs { float4* row_part[2]; float* row_ent; unsigned int* done; unsigned long long* queue; size_t bytes; };
+static LayersWs carve_layers(const structkv_config& cfg, int max_layers, void* base) {
+  LayersWs w{};
+  char* p = (char*)base;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* r = p ? (void*)(p + off) : nullptr;
+    off += align_up(bytes, 256);
+    return r;
+  };
+  const size_t rows_pad = (size_t)rows_pad_of(cfg);
+  w.done = (unsigned int*)take(256);
+  w.queue = (unsigned long long*)take((size_t)max_layers * kQueueUnits * sizeof(unsigned long long));   // follows `done`: one memset
+  for (int i = 0; i < 2; ++i) w.row_part[i] = (float4*)take((size_t)kMaxParts * rows_pad * sizeof(float4));
+  w.row_ent = (float*)take((size_t)max_layers * rows_pad * sizeof(float));
+  w.bytes = off;
+  return w;
+}
+}  // namespace skv
+
+size_t structkv_layers_workspace_bytes(const structkv_config* cfg, int max_layers) {
+  if (!cfg || !config_ok(*cfg) || !config_supported(*cfg) || max_layers < 1 || max_layers > 65536) return 0;
+  return carve_layers(*cfg, max_layers, nullptr).bytes;
+}
+
+structkv_status structkv_score_layers(structkv_ctx* ctx, int n_layers, const void* const* q_windows,
+                                      const void* const* ks, long long k_stride_head,
+                                      long long k_stride_token, int n_keys, const float* scales, float lambda,
+                                      float* s_out, long long s_layer_stride, float* c_inout,
+                                      float* head_cols_out, long long head_cols_layer_stride,
+                                      float* metrics_out, void* layers_workspace,
+                                      size_t layers_workspace_bytes, void* stream) {
+  if (!ctx || !q_windows || !ks || !scales || !s_out || !head_cols_out || !metrics_out)
+    return STRUCTKV_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > 65536) return STRUCTKV_ERR_INVALID_ARG;
+  Ctx& c = ctx->c;
+  const structkv_config& cfg = c.cfg;
+  const int esz = cfg.dtype == STRUCTKV_BF16 ? 2 : 4;
+  if (n_keys < cfg.window || n_keys > cfg.max_seq || !std::isfinite(lambda)) return STRUCTKV_ERR_INVALID_ARG;
+  if (k_stride_token < cfg.head_dim || k_stride_head < 0) return STRUCTKV_ERR_INVALID_ARG;
+  if ((k_stride_token * esz) % 16 || (k_stride_head * esz) % 16) return STRUCTKV_ERR_INVALID_ARG;
+  if (s_layer_stride < n_keys || head_cols_layer_stride < (long long)cfg.n_q_heads * n_keys)
+    return STRUCTKV_ERR_INVALID_ARG;
+  if (((uintptr_t)s_out % 4) || ((uintptr_t)metrics_out % 4) || ((uintptr_t)c_inout % 4) ||
+      ((uintptr_t)head_cols_out % 4))
+    return STRUCTKV_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!q_windows[l] || !ks[l] || ((uintptr_t)q_windows[l] % 16) || ((uintptr_t)ks[l] % 16) ||
+        !std::isfinite(scales[l]))
+      return STRUCTKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  auto args_of = [&](int l) {
+    ScoreArgs a;
+    a.q = q_windows[l]; a.k = ks[l];
+    a.k_stride_head = k_stride_head; a.k_stride_token = k_stride_token;
+    a.n_keys = n_keys; a.scale = scales[l];
+    a.batch = 1; a.total_keys = n_keys; a.cu_seqlens = nullptr;
+    a.cols = head_cols_out + (size_t)l * head_cols_layer_stride;
+    a.col_stride = n_keys;
+    return a;
+  };
+  ScoreArgs probe = args_of(0);
+  if (cfg.dtype != STRUCTKV_BF16 || !tc_supported(c, probe)) {
+    // the CUDA-core scorer has no interleaved form: one layer after the other, same results
+    for (int l = 0; l < n_layers; ++l) {
+      const structkv_status s = structkv_score_layer(
+          ctx, q_windows[l], ks[l], k_stride_head, k_stride_token, n_keys, scales[l], lambda,
+          s_out + (size_t)l * s_layer_stride, c_inout, head_cols_out + (size_t)l * head_cols_layer_stride,
+          metrics_out + 3 * l, STRUCTKV_FLAG_NO_HEAD_STATS, stream);
+      if (s != STRUCTKV_OK) return s;
+    }
+    return STRUCTKV_OK;
+  }
+  const size_t need = carve_layers(cfg, n_layers, nullptr).bytes;
+  if (!layers_workspace || layers_workspace_bytes < need || ((uintptr_t)layers_workspace % 256) != 0)
+    return STRUCTKV_ERR_WORKSPACE;
+  const LayersWs lw = carve_layers(cfg, n_layers, layers_workspace);
+  // completion counters and every layer's own ticket counters start from zero
+  if (cudaMemsetAsync(lw.done, 0, 256 + (size_t)n_layers * kQueueUnits * sizeof(unsigned long long), st) != cudaSuccess)
+    return STRUCTKV_ERR_CUDA;
+
+  // Stream order: P1(0), then for every layer l: P1(l + 1), P2(l).  P2(l) waits for the completion
+  // counter of P1(l), which finished while P1(l + 1) ran, instead of for the whole kernel before it;
+  // P1(l + 2) overwrites the row statistics P2(l) reads only after P2(l), the kernel before it in
+  // the stream, has completed.  Two statistics buffers and two counters alternate.
+  Ctx view = c;
+  auto launch = [&](int l, int pass) {
+    view.ws.row_part = lw.row_part[l & 1];
+    view.ws.row_ent = lw.row_ent + (size_t)l * c.rows_pad;
+    ScoreArgs a = args_of(l);
+    a.inputs_ready = true;
+    a.done = lw.done + (l & 1);
+    a.done_round = l / 2 + 1;
+    a.queue = lw.queue + (size_t)l * kQueueUnits;
+    int parts = 0;
+    return launch_score_tc(view, a, &parts, pass, st) == cudaSuccess;
+  };
+  bool ok = launch(0, 1);
+  for (int l = 0; ok && l < n_layers; ++l) {
+    if (l + 1 < n_layers) ok = launch(l + 1, 1);
+    ok = ok && launch(l, 2);
+  }
+  if (!ok) return STRUCTKV_ERR_CUDA;
+  return launch_reduce_layers(c, head_cols_out, head_cols_layer_stride, n_keys, n_keys, n_layers, lambda, s_out,
+                              s_layer_stride, c_inout, lw.row_ent, metrics_out, st) == cudaSuccess
+             ? STRUCTKV_OK
+             : STRUCTKV_ERR_CUDA;
+}
+
 structkv_status structkv_select_batch(structkv_ctx* ctx, const float* scores, const int* cu_seqlens,
                                       const int* budgets, int batch, int window, int* idx_out,
                                       long long idx_stride, void* stream) {

@@ -67,6 +67,12 @@ struct ScoreArgs {
   const int* cu_seqlens;    // host, [batch + 1] first key of every sequence in the packed K; NULL = plain call
   float scale;
   bool inputs_ready = false; // q and k are complete and visible: nothing in flight on the stream writes them
+  // completion counter of pass 1 (device, or NULL) and how many pass-1 launches, this one included,
+  // have used it since it was zeroed: pass 2 of the same layer waits for done_round * grid
+  unsigned int* done = nullptr;
+  int done_round = 0;
+  // ticket counters for this launch alone ([kQueueUnits], zero), or NULL for the context's shared ones
+  unsigned long long* queue = nullptr;
   float* cols;              // [H][col_stride] pooled per-head attention (output of pass 2)
   long long col_stride;
 };
@@ -95,6 +101,11 @@ cudaError_t launch_finalize_rows(const Ctx& ctx, int parts, cudaStream_t st);
 cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long col_stride, int n, float lambda,
                                  float* s_out, float* c_inout, bool with_head_stats, float* metrics,
                                  cudaStream_t st);
+// The same for n_layers layers in one launch: S^(l) rows s_stride apart, C carried from layer to
+// layer, entropies from row_ent[l][rows_pad]; metrics [n_layers][3] with NaN for sparsity / variance.
+cudaError_t launch_reduce_layers(const Ctx& ctx, const float* cols, long long layer_stride, long long col_stride,
+                                 int n, int n_layers, float lambda, float* s_out, long long s_stride,
+                                 float* c_inout, const float* row_ent, float* metrics, cudaStream_t st);
 
 // Eq. 5-6 for n_layers layers at once from their pooled per-head attention: writes metrics[l][1..2].
 cudaError_t launch_head_stats_batch(const Ctx& ctx, const float* cols, long long layer_stride, long long col_stride,

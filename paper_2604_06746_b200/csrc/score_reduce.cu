@@ -143,6 +143,78 @@ reduce_finish(const float* __restrict__ cols, long long col_stride, int H, int n
   metrics[2] = var / (float)H;
 }
 
+// reduce_finish for several layers at once (the layers' scorer passes have all run): per layer l
+// S^(l) = sum over heads, in reduce_finish's order, C <- lambda C + S^(l) carried in registers from
+// layer to layer, and, in block l, the layer's entropy; sparsity and variance are left as NaN
+// (they come from head_stats).  Every bit equals what a chain of reduce_finish launches gives.
+template <int VEC>
+__global__ void __launch_bounds__(kRcThreads)
+reduce_layers(const float* __restrict__ cols, long long layer_stride, long long col_stride, int H, int n,
+              int n_layers, float lambda, float* __restrict__ s_out, long long s_stride,
+              float* __restrict__ c_inout, const float* __restrict__ row_ent, int rows_pad, int rows_pg_pad,
+              int rows_pg, int n_valid, float* __restrict__ metrics) {
+  __shared__ float red[33];
+  pdl_trigger();
+  pdl_wait();
+  if (VEC == 4) {
+    __shared__ float4 part[3][64];
+    const int lane_j = threadIdx.x & 63, grp = threadIdx.x >> 6;
+    const int j4 = (blockIdx.x * 64 + lane_j) * 4;
+    const int h_per = (H + 3) / 4, h_lo = grp * h_per, h_hi = min(H, h_lo + h_per);
+    float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (grp == 0 && j4 < n && c_inout) c = *reinterpret_cast<const float4*>(c_inout + j4);
+    for (int l = 0; l < n_layers; ++l) {
+      const float* cl = cols + (size_t)l * layer_stride;
+      float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j4 < n) {
+#pragma unroll 4
+        for (int h = h_lo; h < h_hi; ++h) {
+          const float4 v = *reinterpret_cast<const float4*>(cl + (size_t)h * col_stride + j4);
+          s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+      }
+      if (grp > 0) part[grp - 1][lane_j] = s;
+      __syncthreads();
+      if (grp == 0 && j4 < n) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+          const float4 o = part[k][lane_j];
+          s.x += o.x; s.y += o.y; s.z += o.z; s.w += o.w;
+        }
+        *reinterpret_cast<float4*>(s_out + (size_t)l * s_stride + j4) = s;
+        c.x = fmaf(lambda, c.x, s.x); c.y = fmaf(lambda, c.y, s.y);
+        c.z = fmaf(lambda, c.z, s.z); c.w = fmaf(lambda, c.w, s.w);
+      }
+      __syncthreads();                               // part[] is reused by the next layer
+    }
+    if (grp == 0 && j4 < n && c_inout) *reinterpret_cast<float4*>(c_inout + j4) = c;
+  } else if (blockIdx.x * kRcThreads + threadIdx.x < n) {
+    const int j = blockIdx.x * kRcThreads + threadIdx.x;
+    float c = c_inout ? c_inout[j] : 0.f;
+    for (int l = 0; l < n_layers; ++l) {
+      const float* cl = cols + (size_t)l * layer_stride;
+      float s = 0.f;
+      for (int h = 0; h < H; ++h) s += cl[(size_t)h * col_stride + j];
+      s_out[(size_t)l * s_stride + j] = s;
+      c = fmaf(lambda, c, s);
+    }
+    if (c_inout) c_inout[j] = c;
+  }
+  // blocks walk over the layers for the entropies (there may be fewer blocks than layers)
+  for (int l = blockIdx.x; l < n_layers; l += gridDim.x) {
+    float ent = 0.f;
+    for (int r = threadIdx.x; r < rows_pad; r += kRcThreads)
+      if ((r % rows_pg_pad) < rows_pg) ent += row_ent[(size_t)l * rows_pad + r];
+    const float tot = block_sum_1024(ent, red);
+    if (threadIdx.x == 0) {
+      metrics[l * 3 + 0] = tot / (float)n_valid;
+      metrics[l * 3 + 1] = __int_as_float(0x7fc00000);
+      metrics[l * 3 + 2] = __int_as_float(0x7fc00000);
+    }
+    __syncthreads();
+  }
+}
+
 // Per head: sum of squared deviations from 1/n (Eq. 6: the pooled vector sums to 1, so 1/n is its
 // mean; summing deviations instead of squares keeps near-uniform attention from cancelling) and
 // the mass of the k_rho largest entries (Eq. 5) of the pooled attention vector.  A cluster of
@@ -379,6 +451,23 @@ static cudaError_t launch_head_stats(const float* cols, long long layer_stride, 
   if ((long long)n_layers * H >= 2ll * sm_count)
     return launch_head_stats_cl<1>(cols, layer_stride, col_stride, n_layers, H, n, k_rho, head_part, st);
   return launch_head_stats_cl<kHsCluster>(cols, layer_stride, col_stride, n_layers, H, n, k_rho, head_part, st);
+}
+
+cudaError_t launch_reduce_layers(const Ctx& ctx, const float* cols, long long layer_stride, long long col_stride,
+                                 int n, int n_layers, float lambda, float* s_out, long long s_stride,
+                                 float* c_inout, const float* row_ent, float* metrics, cudaStream_t st) {
+  const int H = ctx.cfg.n_q_heads;
+  const int rows_pg_pad = ctx.rows_pad / ctx.cfg.n_kv_heads;
+  const int rows_pg = (H / ctx.cfg.n_kv_heads) * ctx.cfg.window;
+  const bool vec = n % 4 == 0 && col_stride % 4 == 0 && layer_stride % 4 == 0 && s_stride % 4 == 0 &&
+                   ((uintptr_t)cols % 16) == 0 && ((uintptr_t)s_out % 16) == 0 && ((uintptr_t)c_inout % 16) == 0;
+  if (vec)
+    return launch_pdl(reduce_layers<4>, dim3((n / 4 + 63) / 64), dim3(kRcThreads), 0, st, cols, layer_stride,
+                      col_stride, H, n, n_layers, lambda, s_out, s_stride, c_inout, row_ent, ctx.rows_pad,
+                      rows_pg_pad, rows_pg, ctx.rows, metrics);
+  return launch_pdl(reduce_layers<1>, dim3((n + kRcThreads - 1) / kRcThreads), dim3(kRcThreads), 0, st, cols,
+                    layer_stride, col_stride, H, n, n_layers, lambda, s_out, s_stride, c_inout, row_ent,
+                    ctx.rows_pad, rows_pg_pad, rows_pg, ctx.rows, metrics);
 }
 
 cudaError_t launch_reduce_finish(const Ctx& ctx, const float* cols, long long col_stride, int n, float lambda,

@@ -62,6 +62,12 @@ struct TcParams {
   // key tiles of its unit from it until the unit has none left.  The counters only ever grow;
   // a ticket is read modulo the number of tickets one launch draws (SeqDesc::period).
   unsigned long long* queue;
+  int use_tickets;                     // pass 2: draw tiles from the counters (else a fixed split like pass 1's)
+  // Completion counter of pass 1 (or NULL): every pass-1 CTA adds one once its row statistics are
+  // stored; pass 2 then waits for `done_target` instead of for the kernel before it in the stream,
+  // which lets a caller put the NEXT layer's pass 1 between the two passes of a layer.
+  unsigned int* done;
+  unsigned int done_target;
   float4* row_part;                    // pass 1 out, pass 2 in: [segs][n_seq][rows_pad] (ref, Z, U, -)
   float* row_ent;                      // pass 2 out (segment 0 only): [n_seq][rows_pad] entropy of each score row, nats
   float* cols;                         // pass 2 out [H][col_stride], sequence b at column key0_b
@@ -379,7 +385,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
   // end of the sequence: the tiles pass 1 touched last are the ones still in L2.
   const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
   const int n_items = PASS == 1 ? (n_tiles + 1) / 2 : n_tiles;
-  const int t_lo = (int)((long long)seg * n_items / segs);          // pass 1: first pair of this CTA
+  const int t_lo = (int)((long long)seg * n_items / segs);          // fixed split: first item of this CTA
   const int n_static = (int)((long long)(seg + 1) * n_items / segs) - t_lo;
   const int units_per_seq = p.n_rb * (p.rows_pad / p.rows_pg_pad);
   unsigned long long* const ticket = p.queue + (size_t)sq * kQueueUnits + unit;
@@ -424,7 +430,8 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       // first ticket at once: its latency hides behind the Q load
-      unsigned long long tk = PASS == 2 ? atomicAdd(ticket, 1ull) : 0ull;
+      const bool tickets = PASS == 2 && p.use_tickets;
+      unsigned long long tk = tickets ? atomicAdd(ticket, 1ull) : 0ull;
       mbar_expect_tx(bars + 8 * kBarQ, L::kQBytes);
       const int q_row0 = sq * p.q_rows + g * p.rows_pg + rb * kRowBlock;
       for (int s = 0; s < L::kSub; ++s)
@@ -439,8 +446,9 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
       constexpr int kPerItem = PASS == 1 ? 2 : 1;          // K stages one item occupies
       for (int it = 0;; ++it) {
         int item;
-        if (PASS == 1) {
-          item = it < n_static ? t_lo + it : -1;
+        if (!tickets) {
+          // pass 1 ascending; pass 2 descending, from the end of its share
+          item = it < n_static ? (PASS == 1 ? t_lo + it : t_lo + n_static - 1 - it) : -1;
         } else {
           const int idx = (int)(tk % (unsigned long long)(rb == p.n_rb - 1 ? p.seq[sq].period_last : p.seq[sq].period));
           item = idx < n_items ? n_items - 1 - idx : -1;
@@ -729,6 +737,12 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
           }
         }
       }
+      if (p.done) {
+        // the statistics are visible device-wide before the counter moves
+        __threadfence();
+        asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+        if (threadIdx.x == 64) atomicAdd(p.done, 1u);
+      }
     } else {
       // pass 2.  First the compute threads merge the partial statistics of this block's rows,
       // two threads per row (each takes every other partial, loads batched), then one of them
@@ -751,7 +765,24 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
               *reinterpret_cast<__nv_bfloat16*>(ax + k16_offset(ct, k)) = __float2bfloat16_rn(1.0f);
           }
         }
-        pdl_wait();
+        if (p.done) {
+          // pass 1 of this layer is an earlier launch of the stream: all of its CTAs have started
+          // by the time this kernel runs, so the bounded wait below cannot be a wait for work
+          // that is not scheduled yet
+          if (ct == 0) {
+            const long long t0 = clock64();
+            for (;;) {
+              unsigned int seen;
+              asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.done) : "memory");
+              if (seen >= p.done_target || *abort_flag) break;
+              if ((unsigned long long)(clock64() - t0) > kWaitCycles) { *abort_flag = 1; break; }
+              __nanosleep(200);
+            }
+          }
+          asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+        } else {
+          pdl_wait();
+        }
         const int r = ct & (kRowBlock - 1), hp = ct >> 8;
         const size_t row = row_base + r;
         const int parts = segs;
@@ -778,7 +809,7 @@ tc_score(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUte
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {
               const int sidx = s0 + 2 * b;
-              pv[b] = sidx < parts ? __ldg(&p.row_part[(size_t)sidx * p.rows_all + row])
+              pv[b] = sidx < parts ? __ldcg(&p.row_part[(size_t)sidx * p.rows_all + row])
                                    : make_float4(-INFINITY, 0.f, 0.f, 0.f);
             }
 #pragma unroll
@@ -1073,8 +1104,15 @@ cudaError_t launch_score_tc(Ctx& ctx, const ScoreArgs& a, int* parts_out, int pa
   // CTA of the unit, and tickets are read modulo that number.  A slot whose number changes (another
   // sequence length) starts again from zero; this is settled before pass 1, so that nothing comes
   // between the two passes.
-  p.queue = ctx.ws.queue;
-  if (pass == 1)
+  p.queue = a.queue ? a.queue : ctx.ws.queue;
+  // Two launches must never draw from the same counters at the same time.  With the caller's word
+  // that the inputs are ready, the next layer's kernels may start before this layer's pass 2 has
+  // finished, so the shared counters are used only without that word; a caller that interleaves
+  // layers brings counters of its own for every launch.
+  p.use_tickets = (a.queue != nullptr || !a.inputs_ready) ? 1 : 0;
+  p.done = a.done;
+  p.done_target = (unsigned int)(a.done_round * grid);   // every earlier use of the counter added one per CTA of this grid
+  if (pass == 1 && !a.queue)
     for (int b = 0; b < a.batch; ++b) {
       const unsigned int want[2] = {p.seq[b].period, p.seq[b].period_last};
       const bool stale = (ctx.queue_period[b][0] != 0 && ctx.queue_period[b][0] != want[0]) ||

@@ -52,6 +52,7 @@ class Prefill:
         self.defer = bool(defer_head_stats) and not (flags & binding.FLAG_NO_HEAD_STATS) and n_layers <= 128
         self.head_cols = (torch.empty((n_layers, n_q_heads, seq), dtype=f32, device=dev) if self.defer else None)
         self._stats_done = 0
+        self._layers_ws = None
 
     # -- Algorithm 1 lines 3-6 for one layer
     def score(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, scale: float,
@@ -69,6 +70,26 @@ class Prefill:
         self.ctx.score_layer(q_win, k, scale, self.s_hist[layer], self.metrics[layer],
                              c_inout=self.c_running, lam=self.lam, head_cols_out=head_cols_out,
                              flags=self.flags)
+
+    def score_all(self, layers: Sequence[Dict[str, torch.Tensor]]) -> None:
+        """Algorithm 1 lines 3-6 for resident layers.  Where the pooled per-head attention of every layer
+        is kept anyway (head statistics in one batched call) and the layers' K tensors share one layout,
+        all layers go through one structkv_score_layers call, which interleaves the scorer passes of
+        neighbouring layers; otherwise layer after layer."""
+        L = len(layers)
+        k0 = layers[0]["k"]
+        same = all(t["k"].shape == k0.shape and t["k"].stride() == k0.stride() for t in layers)
+        if not (self.defer and same and L == self.L and self.flags in (0, binding.FLAG_INPUTS_READY)):
+            for l, t in enumerate(layers):
+                self.score(l, t["q_win"], t["k"], t["scale"])
+            return
+        if self._layers_ws is None:
+            self._layers_ws = self.ctx.layers_workspace(self.L)
+        self.c_running.zero_()
+        self._stats_done = 0
+        self.ctx.score_layers([t["q_win"] for t in layers], [t["k"] for t in layers],
+                              [t["scale"] for t in layers], self.s_hist, self.metrics, self.head_cols,
+                              self._layers_ws, c_inout=self.c_running, lam=self.lam)
 
     def finish_scores(self, n_scored: Optional[int] = None) -> None:
         """Sparsity and variance (Eq. 5-6) of the layers scored so far, in one batched call."""
@@ -149,8 +170,7 @@ class Prefill:
     def run(self, layers: Sequence[Dict[str, torch.Tensor]], hidden: Optional[torch.Tensor] = None,
             positions: Optional[torch.Tensor] = None) -> int:
         """Whole path over resident per-layer tensors (dicts with q_win, k, v, scale)."""
-        for l, t in enumerate(layers):
-            self.score(l, t["q_win"], t["k"], t["scale"])
+        self.score_all(layers)
         self.detect_and_select(len(layers))
         self.compact_all_kv(layers)
         if hidden is not None:

@@ -359,3 +359,41 @@ def test_a_captured_layer_can_be_replayed(mods, cuda_device):
             torch.cuda.synchronize()
     assert ctx.poll_device_status() == binding.OK
     ctx.close()
+
+
+@pytest.mark.parametrize("name,seq,n_layers", [("llama32k", 9000 + 41, 7), ("qwen64k", 5000 + 3, 4), ("llama32k", 300, 1)])
+def test_all_layers_in_one_call_equal_the_layer_by_layer_calls(mods, cuda_device, name, seq, n_layers):
+    """structkv_score_layers (first pass of layer l + 1 enqueued between the two passes of layer l, the
+    second pass waiting for a completion counter, one reduce over heads for all layers at the end)
+    gives, bit for bit, what structkv_score_layer gives layer after layer: S, C, pooled per-head
+    attention, entropy; and the call can be repeated on the same workspace."""
+    binding, _ = mods
+    wl = synth.WORKLOADS[name].scaled(seq, n_layers=n_layers, n_hubs=4, budgets=(128,))
+    pl = synth.plan(wl)
+    layers = gpu_layers(wl, pl, cuda_device)
+    H, N, dev = wl.n_q_heads, wl.seq, cuda_device
+    ctx = binding.Context(H, wl.n_kv_heads, wl.head_dim, wl.window, N, torch.bfloat16, dev)
+    f32 = torch.float32
+    s1, s2 = (torch.zeros((n_layers, N), dtype=f32, device=dev) for _ in range(2))
+    m1, m2 = (torch.zeros((n_layers, 3), dtype=f32, device=dev) for _ in range(2))
+    h1, h2 = (torch.zeros((n_layers, H, N), dtype=f32, device=dev) for _ in range(2))
+    c1, c2 = (torch.zeros(N, dtype=f32, device=dev) for _ in range(2))
+    for l, t in enumerate(layers):
+        ctx.score_layer(t["q_win"], t["k"], t["scale"], s1[l], m1[l], c_inout=c1, head_cols_out=h1[l],
+                        flags=binding.FLAG_NO_HEAD_STATS)
+    torch.cuda.synchronize()
+    ws = ctx.layers_workspace(n_layers)
+    for rep in range(3):
+        c2.zero_()
+        ctx.score_layers([t["q_win"] for t in layers], [t["k"] for t in layers], [t["scale"] for t in layers],
+                         s2, m2, h2, ws, c_inout=c2)
+        torch.cuda.synchronize()
+        assert ctx.poll_device_status() == binding.OK
+        assert torch.equal(s1, s2) and torch.equal(h1, h2) and torch.equal(c1, c2), f"repeat {rep}"
+        assert torch.equal(m1[:, 0], m2[:, 0]) and torch.isnan(m2[:, 1:]).all()
+    # a workspace that is too small is refused on the host
+    small = ws[: ws.numel() - 256]
+    with pytest.raises(Exception):
+        ctx.score_layers([t["q_win"] for t in layers], [t["k"] for t in layers], [t["scale"] for t in layers],
+                         s2, m2, h2, small, c_inout=c2)
+    ctx.close()
