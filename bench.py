@@ -38,11 +38,11 @@ SFU_EXP_PER_CLK_PER_SM = 16      # special-function results per clock per SM (cc
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the scorer launches of one layer,
 # from an ncu capture of the current kernels; None = no capture of the current kernels exists.
-NCU_TRAFFIC_BYTES_PER_LAYER = 512.0e6
+NCU_TRAFFIC_BYTES_PER_LAYER = 549.0e6
 NCU_TRAFFIC_NOTE = ("dram read + write of the two tc_score launches of one layer (llama128k shape), single-metric "
                     "ncu captures with the caches left as the previous kernel leaves them: pass 1 reads 269 MB, "
-                    "pass 2 209-211 MB (it starts with the tiles pass 1 asked L2 to keep and finds more than a fifth of K "
-                    "there), 28 + 5 MB written")
+                    "pass 2 252 MB when the next layer's pass 1 ran in between (every layer but the last; 218 MB "
+                    "otherwise: it starts with the tiles pass 1 asked L2 to keep), 28 + 1 MB written")
 
 
 def load_peaks():
