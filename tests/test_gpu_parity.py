@@ -361,12 +361,14 @@ def test_a_captured_layer_can_be_replayed(mods, cuda_device):
     ctx.close()
 
 
-@pytest.mark.parametrize("name,seq,n_layers", [("llama32k", 9000 + 41, 7), ("qwen64k", 5000 + 3, 4), ("llama32k", 300, 1)])
+@pytest.mark.parametrize("name,seq,n_layers", [("llama32k", 9000 + 41, 7), ("qwen64k", 5000 + 3, 4), ("llama32k", 300, 1),
+                                                ("llama32k", 300, 9), ("llama128k", 1200, 12)])
 def test_all_layers_in_one_call_equal_the_layer_by_layer_calls(mods, cuda_device, name, seq, n_layers):
     """structkv_score_layers (first pass of layer l + 1 enqueued between the two passes of layer l, the
     second pass waiting for a completion counter, one reduce over heads for all layers at the end)
     gives, bit for bit, what structkv_score_layer gives layer after layer: S, C, pooled per-head
-    attention, entropy; and the call can be repeated on the same workspace."""
+    attention, entropy; and the call can be repeated on the same workspace.  The short sequences give
+    grids of a few CTAs, so many launches of the call are resident at once."""
     binding, _ = mods
     wl = synth.WORKLOADS[name].scaled(seq, n_layers=n_layers, n_hubs=4, budgets=(128,))
     pl = synth.plan(wl)
