@@ -596,9 +596,11 @@ def workload_config(wl, kv_budget):
                         f"head_dim {wl.head_dim}, seq {wl.seq}, window {wl.window}",
             "kv_budget": kv_budget, "struct_budget": wl.struct_budget(kv_budget),
             "lambda": 0.9, "weights": [0.2, 0.3, 0.5],
-            "l2": "inputs larger than L2 (each layer's K is %.0f MB, read once per step; a step touches "
-                  "%.1f GB of distinct K/V)" % (wl.n_kv_heads * wl.seq * wl.head_dim * esz / 1e6,
-                                                wl.n_layers * 2 * wl.n_kv_heads * wl.seq * wl.head_dim * esz / 1e9)}
+            "scoring": "all resident layers in one structkv_score_layers call (layer by layer where the "
+                       "CUDA-core scorer serves the shape)",
+            "l2": "inputs larger than L2 (each layer's K is %.0f MB and no layer is touched twice in a step; a "
+                  "step touches %.1f GB of distinct K/V)" % (wl.n_kv_heads * wl.seq * wl.head_dim * esz / 1e6,
+                                                           wl.n_layers * 2 * wl.n_kv_heads * wl.seq * wl.head_dim * esz / 1e9)}
 
 
 def other_configs(dev, peaks, sm_mhz, min_seconds, skip):
