@@ -53,6 +53,7 @@ class Prefill:
         self.head_cols = (torch.empty((n_layers, n_q_heads, seq), dtype=f32, device=dev) if self.defer else None)
         self._stats_done = 0
         self._layers_ws = None
+        self._side = None
 
     # -- Algorithm 1 lines 3-6 for one layer
     def score(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, scale: float,
@@ -102,10 +103,19 @@ class Prefill:
     def detect_and_select(self, n_scored: Optional[int] = None) -> int:
         L = self.L if n_scored is None else n_scored
         self.finish_scores(L)
-        self.pivot, self.transition = self.ctx.pivot(self.metrics[:L], self.weights, self.l_limit)
+        # The per-layer selections (Eq. 13) do not depend on the pivot: they are enqueued first, and the
+        # metric table travels to the host on a side stream meanwhile, so the device is not idle while
+        # the host evaluates Eq. 7-9.
+        main = torch.cuda.current_stream(self.device)
+        if self._side is None:
+            self._side = torch.cuda.Stream(device=self.device)
+        ready = torch.cuda.Event()
+        ready.record(main)
+        self._side.wait_event(ready)
+        self.ctx.select(self.s_hist[:L], self.kv_budget, self.w, self.i_kv[:L])
+        self.pivot, self.transition = self.ctx.pivot(self.metrics[:L], self.weights, self.l_limit, stream=self._side)
         self.ctx.accumulate(self.s_hist, self.pivot, self.lam, self.c_star)
         self.ctx.select(self.c_star, self.struct_budget, self.w, self.i_struct)
-        self.ctx.select(self.s_hist[:L], self.kv_budget, self.w, self.i_kv[:L])
         return self.pivot
 
     # -- Algorithm 1 line 17 for one layer
