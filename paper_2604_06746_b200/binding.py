@@ -145,6 +145,25 @@ def score_layer_static(n_q_heads: int, n_kv_heads: int, head_dim: int, window: i
                "structkv_score_layer_static")
 
 
+class LayerSources:
+    """Host-side argument block for ``Context.compact_layers`` (pointers and layout of the sources)."""
+
+    def __init__(self, srcs: Sequence[torch.Tensor]):
+        s0 = srcs[0]
+        assert all(t.shape == s0.shape and t.stride() == s0.stride() and t.dtype == s0.dtype for t in srcs)
+        row_elems = 1
+        for sdim in s0.shape[2:]:
+            row_elems *= sdim
+        self.keep = list(srcs)                       # the tensors must outlive the block
+        self.n_layers = len(srcs)
+        self.elem_size = s0.element_size()
+        self.ptrs = (_vp * self.n_layers)(*[t.data_ptr() for t in srcs])
+        self.slab_stride_bytes = s0.stride(0) * self.elem_size
+        self.row_stride_bytes = s0.stride(1) * self.elem_size
+        self.row_bytes = row_elems * self.elem_size
+        self.n_slabs, self.n_rows = s0.shape[0], s0.shape[1]
+
+
 class Context:
     """Owns the library context and (through torch) its device workspace."""
 
@@ -297,23 +316,26 @@ class Context:
                                     row_elems * es, src.shape[0], src.shape[1], idx.data_ptr(),
                                     idx.numel(), dst.data_ptr(), _stream(stream)), "structkv_compact")
 
-    def compact_layers(self, srcs: Sequence[torch.Tensor], idx: torch.Tensor, dst: torch.Tensor,
+    @staticmethod
+    def layer_sources(srcs: Sequence[torch.Tensor]) -> "LayerSources":
+        """The argument block of ``compact_layers`` for a fixed list of source tensors (same shape,
+        strides and dtype), checked and marshalled once: a caller that gathers from the same tensors
+        many times keeps it and spares the per-call marshalling."""
+        return LayerSources(srcs)
+
+    def compact_layers(self, srcs, idx: torch.Tensor, dst: torch.Tensor,
                        stream: Optional[torch.cuda.Stream] = None) -> None:
         """structkv_compact_layers: every ``srcs[l] [n_slabs, n_rows, row...]`` (same shape and strides)
-        gathered at ``idx[l]`` into ``dst[l] [n_slabs, n_idx, row...]`` by one launch."""
-        L = len(srcs)
-        s0 = srcs[0]
+        gathered at ``idx[l]`` into ``dst[l] [n_slabs, n_idx, row...]`` by one launch.  ``srcs`` is a list of
+        tensors or the ``LayerSources`` made from one."""
+        ls = srcs if isinstance(srcs, LayerSources) else LayerSources(srcs)
+        L = ls.n_layers
         assert idx.dtype == torch.int32 and idx.dim() == 2 and idx.shape[0] == L and idx.stride(1) == 1
         assert dst.shape[0] == L and dst[0].is_contiguous()
-        assert all(t.shape == s0.shape and t.stride() == s0.stride() and t.dtype == s0.dtype for t in srcs)
-        row_elems = 1
-        for sdim in s0.shape[2:]:
-            row_elems *= sdim
-        es = s0.element_size()
-        ptrs = (_vp * L)(*[t.data_ptr() for t in srcs])
-        _check(lib.structkv_compact_layers(self._h, ptrs, L, s0.stride(0) * es, s0.stride(1) * es, row_elems * es,
-                                           s0.shape[0], s0.shape[1], idx.data_ptr(), idx.stride(0), idx.shape[1],
-                                           dst.data_ptr(), dst.stride(0) * es, _stream(stream)),
+        _check(lib.structkv_compact_layers(self._h, ls.ptrs, L, ls.slab_stride_bytes, ls.row_stride_bytes,
+                                           ls.row_bytes, ls.n_slabs, ls.n_rows, idx.data_ptr(), idx.stride(0),
+                                           idx.shape[1], dst.data_ptr(), dst.stride(0) * ls.elem_size,
+                                           _stream(stream)),
                "structkv_compact_layers")
 
     def group_saliency(self, head_cols: torch.Tensor, out: torch.Tensor,

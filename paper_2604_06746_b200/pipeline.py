@@ -54,6 +54,7 @@ class Prefill:
         self._stats_done = 0
         self._layers_ws = None
         self._side = None
+        self._kv_sources = None
 
     # -- Algorithm 1 lines 3-6 for one layer
     def score(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, scale: float,
@@ -134,9 +135,14 @@ class Prefill:
         """Algorithm 1 line 17 for resident layers: one launch for all of them when every layer keeps
         K and V in one joint allocation, else one gather per layer."""
         if self.keep_kv and len(layers) <= 128 and all("kv" in t for t in layers):
-            self.ctx.compact_layers([t["kv"].view(2 * self.Hkv, t["kv"].shape[2], self.d) for t in layers],
-                                    self.i_kv[:len(layers)],
-                                    self.kv_out[:len(layers)].view(len(layers), 2 * self.Hkv, self.kv_budget, self.d))
+            # the sources' pointers and layout are marshalled once per set of tensors, so that the launch
+            # is not held up by host work after the selections
+            key = tuple(t["kv"].data_ptr() for t in layers)
+            if self._kv_sources is None or self._kv_sources[0] != key:
+                self._kv_sources = (key, self.ctx.layer_sources(
+                    [t["kv"].view(2 * self.Hkv, t["kv"].shape[2], self.d) for t in layers]))
+                self._kv_dst = self.kv_out[:len(layers)].view(len(layers), 2 * self.Hkv, self.kv_budget, self.d)
+            self.ctx.compact_layers(self._kv_sources[1], self.i_kv[:len(layers)], self._kv_dst)
             return
         for l, t in enumerate(layers):
             if "v" in t:
